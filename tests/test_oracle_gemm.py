@@ -1,0 +1,113 @@
+"""Pins for the oracle's FP8 GEMM: exact rational brute force on tiny inputs,
+numpy's float64 matmul where the sum is exact, structured operands with closed
+forms, and special-value propagation."""
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import E4M3, E5M2
+
+
+def _finite_codes(rng, fmt, shape):
+    c = rng.integers(0, 256, size=shape, dtype=np.uint16).astype(np.uint8)
+    t = oracle.decode_table(fmt)
+    bad = ~np.isfinite(t[c])
+    c[bad] = 0x38 if fmt == E4M3 else 0x3C        # 1.0
+    return c
+
+
+def _frac_table(fmt):
+    t = oracle.decode_table(fmt)
+    return [Fraction(float(v)) if np.isfinite(v) else None for v in t]
+
+
+ROLES = [(E4M3, E4M3), (E5M2, E4M3), (E4M3, E5M2)]     # forward, dgrad, wgrad operand formats
+
+
+@pytest.mark.parametrize("fa,fb", ROLES)
+def test_gemm_equals_exact_rational_brute_force(fa, fb):
+    rng = np.random.default_rng(100 + fa * 2 + fb)
+    M, N, K = 5, 7, 33
+    A = _finite_codes(rng, fa, (M, K))
+    B = _finite_codes(rng, fb, (K, N))
+    ta, tb = _frac_table(fa), _frac_table(fb)
+    sa_inv, sb_inv = np.float32(0.0371), np.float32(1.0 / 3.0)
+    ref, sab = oracle.gemm_rows(A, fa, (K, 1), B, fb, (N, 1), N, K, 0, M, sa_inv, sb_inv)
+    alpha = Fraction(float(sa_inv)) * Fraction(float(sb_inv))
+    for i in range(M):
+        for j in range(N):
+            exact = sum(ta[A[i, k]] * tb[B[k, j]] for k in range(K)) * alpha
+            exabs = sum(abs(ta[A[i, k]] * tb[B[k, j]]) for k in range(K)) * alpha
+            assert abs(Fraction(float(ref[i, j])) - exact) <= Fraction(1, 10 ** 14) * exabs
+            assert abs(Fraction(float(sab[i, j])) - exabs) <= Fraction(1, 10 ** 14) * exabs
+            # the 128-bit fixed-point dot product is the exact sum
+            integer, ue = oracle.dot_exact(A[i, :], fa, B[:, j].copy(), fb)
+            assert Fraction(integer) * Fraction(2) ** ue * alpha == exact
+
+
+def test_e4m3_gemm_is_exact_and_equals_numpy_float64_matmul():
+    rng = np.random.default_rng(5)
+    M, N, K = 16, 24, 512
+    A = _finite_codes(rng, E4M3, (M, K))
+    B = _finite_codes(rng, E4M3, (K, N))
+    t = oracle.decode_table(E4M3)
+    ref, sab = oracle.gemm_rows(A, E4M3, (K, 1), B, E4M3, (N, 1), N, K, 0, M, 1.0, 1.0)
+    # every product is a multiple of 2^-18 and the sum stays far below 2^53 units: any order is exact
+    assert np.array_equal(ref, t[A] @ t[B])
+    assert np.array_equal(sab, np.abs(t[A]) @ np.abs(t[B]))
+
+
+@pytest.mark.parametrize("fa,fb", ROLES)
+def test_operand_layouts_give_the_same_numbers(fa, fb):
+    rng = np.random.default_rng(9)
+    M, N, K = 6, 10, 40
+    A = _finite_codes(rng, fa, (M, K))
+    B = _finite_codes(rng, fb, (K, N))
+    base, _ = oracle.gemm_rows(A, fa, (K, 1), B, fb, (N, 1), N, K, 0, M, 0.5, 0.25)
+    At = np.ascontiguousarray(A.T)          # stored [K, M]: the row index is the contiguous one
+    Bt = np.ascontiguousarray(B.T)          # stored [N, K]: the contraction index is the contiguous one
+    alt, _ = oracle.gemm_rows(At, fa, (1, M), Bt, fb, (1, K), N, K, 0, M, 0.5, 0.25)
+    assert np.array_equal(base, alt)
+    ii = np.array([0, 5, 3, 2], dtype=np.int64)
+    jj = np.array([9, 0, 4, 4], dtype=np.int64)
+    s, _ = oracle.gemm_samples(At, fa, (1, M), Bt, fb, (1, K), K, ii, jj, 0.5, 0.25)
+    assert np.array_equal(s, base[ii, jj])
+    part, _ = oracle.gemm_rows(A, fa, (K, 1), B, fb, (N, 1), N, K, 2, 5, 0.5, 0.25, threads=2)
+    assert np.array_equal(part, base[2:5])
+
+
+def test_structured_operands_closed_forms():
+    rng = np.random.default_rng(12)
+    K = 64
+    A = _finite_codes(rng, E5M2, (8, K))
+    ta = oracle.decode_table(E5M2)
+    one, zero = 0x38, 0x00
+    eye = np.where(np.eye(K, dtype=bool), one, zero).astype(np.uint8)
+    ref, _ = oracle.gemm_rows(A, E5M2, (K, 1), eye, E4M3, (K, 1), K, K, 0, 8, 0.125, 2.0)
+    assert np.array_equal(ref, ta[A] * 0.25)                 # identity B returns the decoded A, unscaled once
+    ones = np.full((K, 1), one, dtype=np.uint8)
+    ref, sab = oracle.gemm_rows(A, E5M2, (K, 1), ones, E4M3, (1, 1), 1, K, 0, 8, 1.0, 1.0)
+    assert np.allclose(ref[:, 0], ta[A].sum(axis=1), rtol=1e-15, atol=0)
+    assert np.allclose(sab[:, 0], np.abs(ta[A]).sum(axis=1), rtol=1e-15, atol=0)
+    ref, sab = oracle.gemm_rows(A, E5M2, (K, 1), eye, E4M3, (K, 1), K, 0, 0, 8, 1.0, 1.0)   # K = 0
+    assert np.all(ref == 0) and np.all(sab == 0)
+
+
+def test_special_codes_propagate():
+    K = 8
+    one = 0x38
+    A = np.full((1, K), 0x3C, dtype=np.uint8)        # E5M2 ones
+    B = np.full((K, 1), one, dtype=np.uint8)
+    A[0, 3] = 0x7C                                   # +Inf
+    ref, _ = oracle.gemm_rows(A, E5M2, (K, 1), B, E4M3, (1, 1), 1, K, 0, 1, 1.0, 1.0)
+    assert ref[0, 0] == np.inf
+    B[3, 0] = 0x00                                   # Inf * 0
+    ref, _ = oracle.gemm_rows(A, E5M2, (K, 1), B, E4M3, (1, 1), 1, K, 0, 1, 1.0, 1.0)
+    assert np.isnan(ref[0, 0])
+    A[0, 3] = 0x3C
+    B[5, 0] = 0x7F                                   # E4M3 NaN
+    ref, _ = oracle.gemm_rows(A, E5M2, (K, 1), B, E4M3, (1, 1), 1, K, 0, 1, 1.0, 1.0)
+    assert np.isnan(ref[0, 0])
+    assert oracle.dot_exact(A[0], E5M2, B[:, 0].copy(), E4M3) is None
