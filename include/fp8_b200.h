@@ -1,0 +1,154 @@
+/*
+ * fp8_b200 — C ABI of the B200 (sm_100a) FP8 hot path of
+ * "FP8 Formats for Deep Learning" (arXiv 2209.05433).
+ *
+ * Conventions shared by every call
+ *   - Every pointer whose name ends in _dev, and every tensor pointer (x, c,
+ *     out, A, B, D), is a DEVICE pointer owned by the caller.  The library
+ *     never allocates or frees device memory and keeps no per-call state.
+ *   - Scalars that flow between calls (amax, scale, scale_inv) live in device
+ *     memory, so amax -> scale -> quantize -> gemm chain on one stream with no
+ *     host synchronisation.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls only enqueue work and return; argument errors are found on the
+ *     host before anything is launched.
+ *   - The return value is a status code; nothing aborts or throws.  A launch
+ *     failure is reported as FP8_ERR_CUDA.  A device-side wait that ran out of
+ *     patience (never expected) is latched and read by fp8_async_status().
+ *   - bf16 tensors are arrays of 16-bit patterns (the upper half of binary32);
+ *     FP8 tensors are arrays of 8-bit codes in the paper's S.E.M layout.
+ */
+#ifndef FP8_B200_H
+#define FP8_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FP8_OK = 0,
+    FP8_ERR_NULL = 1,        /* a required pointer is NULL */
+    FP8_ERR_ENUM = 2,        /* an enum argument is out of range */
+    FP8_ERR_SHAPE = 3,       /* negative size, or a leading dimension smaller than the row */
+    FP8_ERR_ALIGN = 4,       /* GEMM operand base or leading dimension not 16-byte aligned */
+    FP8_ERR_UNSUPPORTED = 5, /* a size beyond what the launch geometry can address */
+    FP8_ERR_CUDA = 6,        /* the CUDA runtime / driver reported an error */
+    FP8_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (see fp8_async_status) */
+} fp8_status;
+
+/* The two encodings of Section 3 / Table 1. */
+typedef enum { FP8_E4M3 = 0, FP8_E5M2 = 1 } fp8_format;
+/* The wider type a tensor is converted from / to (Section 2). */
+typedef enum { FP8_F32 = 0, FP8_BF16 = 1 } fp8_wide;
+/* Section 2: overflow saturates to the maximum finite value (default), or, in the
+ * non-saturating mode, becomes NaN (E4M3, which has no infinity) / Inf (E5M2). */
+typedef enum { FP8_SATURATE = 0, FP8_NOSAT = 1 } fp8_overflow;
+/* Which index of a GEMM operand is contiguous in memory. */
+typedef enum { FP8_MAJOR_K = 0, FP8_MAJOR_MN = 1 } fp8_major;
+
+/*
+ * fp8_amax — maximum magnitude of a tensor (Section 2: the quantity the scale
+ * factor is chosen from).
+ *   x         device, n elements of type t, any element-aligned address.
+ *   amax_dev  device, one float, OVERWRITTEN with max_i |x_i| (+0 when n == 0).
+ *             If any element is NaN the result is NaN (pattern 0x7FC00000);
+ *             otherwise an infinity gives +Inf.  The result is exact and does
+ *             not depend on reduction order.
+ */
+fp8_status fp8_amax(const void* x, fp8_wide t, size_t n, float* amax_dev, void* stream);
+
+/*
+ * fp8_scale_from_amax — Section 2: the scale factor that moves the tensor's
+ * maximum magnitude onto the format's maximum (Table 1: 448 / 57344).
+ *   scale = fmax / amax (binary32 division); amax of 0, NaN or Inf gives 1; a
+ *   quotient that overflows is clamped to the largest finite binary32.
+ *   scale_inv = 1 / scale.  All three pointers are device floats.
+ */
+fp8_status fp8_scale_from_amax(const float* amax_dev, fp8_format f,
+                               float* scale_dev, float* scale_inv_dev, void* stream);
+
+/*
+ * fp8_quantize — Section 2: multiply by the per-tensor scale factor, convert to
+ * FP8 (Table 1 encodings) with round-to-nearest-even.
+ *   out_i = encode_f( binary32(x_i) * scale ), the product rounded to binary32
+ *   first.  Special values convert to special values in both overflow modes:
+ *   NaN -> sign|0x7F; +-Inf -> E4M3 sign|0x7F (NaN), E5M2 sign|0x7C (Inf); this
+ *   rule is applied to the scaled value.  Finite overflow follows `o`.  The sign
+ *   of zero and of values that round to zero is kept.
+ *   x          device, n elements of type t.
+ *   scale_dev  device float, read by the kernel.
+ *   out        device, n bytes.
+ *   amax_dev   NULL, or a device float OVERWRITTEN with amax(x) of the same pass
+ *              (same definition as fp8_amax), for callers that scale with the
+ *              previous step's amax.
+ *   Fast path: x and out both 16-byte aligned; other alignments take a slower
+ *   element-wise path with identical results.
+ */
+fp8_status fp8_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o,
+                        const float* scale_dev, uint8_t* out, float* amax_dev, void* stream);
+
+/*
+ * fp8_dequantize — Section 2: convert back and multiply by the inverse of the
+ * scale factor.  out_i = round_t( decode_f(c_i) * scale_inv ), one binary32
+ * multiply, then round-to-nearest-even to bf16 when t is FP8_BF16.  NaN codes
+ * give NaN (payload unspecified), E5M2 infinities give infinities.
+ */
+fp8_status fp8_dequantize(const uint8_t* c, size_t n, fp8_format f,
+                          const float* scale_inv_dev, void* out, fp8_wide t, void* stream);
+
+/*
+ * fp8_gemm — Sections 2, 3 and 4.1: the matrix multiply on FP8 inputs with a
+ * higher-precision result, unscaled once per dot product.
+ *   D[i,j] = round_out( (sum_k decode_fa(A[i,k]) * decode_fb(B[k,j])) * (sa_inv * sb_inv) )
+ * with binary32 accumulation on the tensor cores.
+ * Operand roles (Section 3: E4M3 for weights and activations, E5M2 for
+ * gradients): forward  fa=E4M3, fb=E4M3;  dgrad  fa=E5M2 (dY), fb=E4M3 (W);
+ * wgrad  fa=E4M3 (X^T), fb=E5M2 (dY).  Any of the four pairs is accepted.
+ *   A   M x K codes.  ma == FP8_MAJOR_K : A[i,k] at A[i*lda + k] (lda >= K);
+ *                     ma == FP8_MAJOR_MN: A[i,k] at A[k*lda + i] (lda >= M).
+ *   B   K x N codes.  mb == FP8_MAJOR_K : B[k,j] at B[j*ldb + k] (ldb >= K);
+ *                     mb == FP8_MAJOR_MN: B[k,j] at B[k*ldb + j] (ldb >= N).
+ *   D   M x N, row-major, D[i,j] at D[i*ldd + j], of type `out` (ldd in elements).
+ *   scale_inv_a_dev / scale_inv_b_dev  device floats (the operands' inverse scales).
+ *   amax_d_dev  NULL, or a device float OVERWRITTEN with amax of D as stored
+ *               (after rounding), same definition as fp8_amax.
+ * Alignment: A, B, D base addresses, lda, ldb (bytes) and ldd*sizeof(out) must
+ * be multiples of 16, else FP8_ERR_ALIGN.  M, N, K are otherwise arbitrary
+ * (edges are zero-filled on load and clipped on store).  M*N == 0 is a no-op
+ * (amax = 0); K == 0 writes zeros.
+ */
+typedef struct {
+    int64_t M, N, K;
+    fp8_format fa, fb;
+    fp8_major ma, mb;
+    int64_t lda, ldb, ldd;
+    fp8_wide out;
+} fp8_gemm_desc;
+
+fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,
+                    const float* scale_inv_a_dev, const float* scale_inv_b_dev,
+                    float* amax_d_dev, void* stream);
+
+/*
+ * fp8_async_status — reads and clears the device-side error latch of the
+ * current device (synchronises the device).  FP8_OK, or FP8_ERR_TIMEOUT if a
+ * kernel gave up on a bounded wait since the last call; *detail (optional, host
+ * pointer) receives a code naming the wait.  Not part of the paper: it exists
+ * so that a pipeline fault ends in an error code instead of a hung GPU.
+ */
+fp8_status fp8_async_status(uint32_t* detail);
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* fp8_status_string(fp8_status s);
+
+/* Number of kernel launches (and memset nodes) the library has enqueued since
+ * it was loaded; host-side counter used by benchmarks to report launch counts. */
+uint64_t fp8_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP8_B200_H */

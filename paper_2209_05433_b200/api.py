@@ -1,0 +1,165 @@
+"""Python binding of the fp8_b200 C ABI (include/fp8_b200.h).
+
+Argument marshalling only: every function checks dtypes, takes `data_ptr()` of
+torch CUDA tensors, passes torch's current stream and calls the entry point of
+the same name in ``libfp8_b200.so``.  There is no fallback: if the library is
+not built, or a call returns a non-zero status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import _build
+
+E4M3, E5M2 = 0, 1            # fp8_format
+F32, BF16 = 0, 1             # fp8_wide
+SATURATE, NOSAT = 0, 1       # fp8_overflow
+MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
+
+EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_dequantize", "fp8_gemm",
+           "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
+
+
+class Fp8Error(RuntimeError):
+    pass
+
+
+class GemmDesc(ctypes.Structure):
+    _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("fa", ctypes.c_int), ("fb", ctypes.c_int), ("ma", ctypes.c_int), ("mb", ctypes.c_int),
+                ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldd", ctypes.c_int64), ("out", ctypes.c_int)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True) -> ctypes.CDLL:
+    """Loads libfp8_b200.so (building it with nvcc when it is missing or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if build_if_missing and _build.is_stale():
+        try:
+            _build.build_library()
+        except Exception as e:
+            if not os.path.exists(path):     # stale is tolerable, missing is not
+                raise Fp8Error("libfp8_b200.so is missing and could not be built: %s" % e) from e
+    if not os.path.exists(path):
+        raise Fp8Error("libfp8_b200.so not found at %s; run `python -m paper_2209_05433_b200._build`" % path)
+    lib = ctypes.CDLL(path)
+    vp, sz, i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+    lib.fp8_amax.restype = i32
+    lib.fp8_amax.argtypes = [vp, i32, sz, vp, vp]
+    lib.fp8_scale_from_amax.restype = i32
+    lib.fp8_scale_from_amax.argtypes = [vp, i32, vp, vp, vp]
+    lib.fp8_quantize.restype = i32
+    lib.fp8_quantize.argtypes = [vp, i32, sz, i32, i32, vp, vp, vp, vp]
+    lib.fp8_dequantize.restype = i32
+    lib.fp8_dequantize.argtypes = [vp, sz, i32, vp, vp, i32, vp]
+    lib.fp8_gemm.restype = i32
+    lib.fp8_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp]
+    lib.fp8_async_status.restype = i32
+    lib.fp8_async_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
+    lib.fp8_status_string.restype = ctypes.c_char_p
+    lib.fp8_status_string.argtypes = [i32]
+    lib.fp8_launch_count.restype = ctypes.c_uint64
+    lib.fp8_launch_count.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _check(status: int, what: str) -> None:
+    if status != 0:
+        raise Fp8Error("%s failed: %s (status %d)" % (what, load().fp8_status_string(status).decode(), status))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _wide_of(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("wide tensors must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _dev(t: torch.Tensor, name: str) -> int:
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor" % name)
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    return t.data_ptr()
+
+
+def _scalar(t: torch.Tensor, name: str) -> int:
+    if t.dtype != torch.float32 or t.numel() != 1:
+        raise TypeError("%s must be a one-element float32 CUDA tensor" % name)
+    return _dev(t, name)
+
+
+def fp8_amax(x: torch.Tensor, amax_out: torch.Tensor) -> None:
+    _check(load().fp8_amax(_dev(x, "x"), _wide_of(x), x.numel(), _scalar(amax_out, "amax_out"), _stream()), "fp8_amax")
+
+
+def fp8_scale_from_amax(amax: torch.Tensor, fmt: int, scale_out: torch.Tensor, scale_inv_out: torch.Tensor) -> None:
+    _check(load().fp8_scale_from_amax(_scalar(amax, "amax"), fmt, _scalar(scale_out, "scale_out"),
+                                      _scalar(scale_inv_out, "scale_inv_out"), _stream()), "fp8_scale_from_amax")
+
+
+def fp8_quantize(x: torch.Tensor, fmt: int, scale: torch.Tensor, out: torch.Tensor,
+                 overflow: int = SATURATE, amax_out: torch.Tensor | None = None) -> None:
+    if out.dtype != torch.uint8 or out.numel() != x.numel():
+        raise TypeError("out must be a uint8 tensor with as many elements as x")
+    _check(load().fp8_quantize(_dev(x, "x"), _wide_of(x), x.numel(), fmt, overflow, _scalar(scale, "scale"),
+                               _dev(out, "out"), None if amax_out is None else _scalar(amax_out, "amax_out"),
+                               _stream()), "fp8_quantize")
+
+
+def fp8_dequantize(codes: torch.Tensor, fmt: int, scale_inv: torch.Tensor, out: torch.Tensor) -> None:
+    if codes.dtype != torch.uint8 or out.numel() != codes.numel():
+        raise TypeError("codes must be uint8 and out must have as many elements")
+    _check(load().fp8_dequantize(_dev(codes, "codes"), codes.numel(), fmt, _scalar(scale_inv, "scale_inv"),
+                                 _dev(out, "out"), _wide_of(out), _stream()), "fp8_dequantize")
+
+
+def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
+             scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, amax_out: torch.Tensor | None = None) -> None:
+    """D[M,N] = (A[M,K] . B[K,N]) * scale_inv_a * scale_inv_b.
+
+    A is a 2-D uint8 tensor stored [M,K] when ``ma == MAJOR_K`` or [K,M] when
+    ``ma == MAJOR_MN``; B is stored [N,K] when ``mb == MAJOR_K`` or [K,N] when
+    ``mb == MAJOR_MN``.  Row pitches are taken from the tensors' strides."""
+    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
+        raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D tensor")
+    for t, name in ((A, "A"), (B, "B"), (D, "D")):
+        if not t.is_cuda or t.stride(1) != 1:
+            raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
+    M, K = (A.shape[0], A.shape[1]) if ma == MAJOR_K else (A.shape[1], A.shape[0])
+    Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
+    if K != Kb or tuple(D.shape) != (M, N):
+        raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
+    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D))
+    _check(load().fp8_gemm(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
+                           _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
+                           None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()), "fp8_gemm")
+
+
+def fp8_async_status() -> tuple[int, int]:
+    """(status, detail) of the device-side error latch; synchronises the device."""
+    detail = ctypes.c_uint32(0)
+    s = load().fp8_async_status(ctypes.byref(detail))
+    return int(s), int(detail.value)
+
+
+def fp8_launch_count() -> int:
+    return int(load().fp8_launch_count())

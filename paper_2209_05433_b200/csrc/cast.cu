@@ -1,0 +1,490 @@
+// amax, scale selection, quantize (wide -> FP8) and dequantize (FP8 -> wide):
+// the memory-bound half of the FP8 hot path (Section 2 of the paper).
+//
+// All four tensor kernels are persistent grid-stride loops over 16-byte items
+// with several independent 128-bit loads in flight per thread; every warp-level
+// load and store instruction covers one contiguous span.  HBM traffic is the
+// algorithmic minimum (each input byte read once, each output byte written once).
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <mutex>
+
+#include "codec.cuh"
+#include "common.cuh"
+
+namespace fp8b200 {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+int sm_count() {
+    static std::mutex mu;
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        cached[dev] = v;
+    }
+    return cached[dev];
+}
+
+constexpr int kWideF32 = 0;
+constexpr int kWideBF16 = 1;
+constexpr int kThreads = 256;
+
+// ---------------------------------------------------------------------------
+// per-item arithmetic
+// ---------------------------------------------------------------------------
+
+// Magnitude bits of one 16-byte item folded into a running maximum.
+// bf16: packed 16-bit maxima (two lanes per word); f32: 32-bit maxima.
+template <int WIDE>
+__device__ __forceinline__ uint32_t fold_abs_max(uint32_t m, const uint4& v) {
+    if (WIDE == kWideBF16) {
+        m = __vmaxu2(m, v.x & 0x7FFF7FFFu);
+        m = __vmaxu2(m, v.y & 0x7FFF7FFFu);
+        m = __vmaxu2(m, v.z & 0x7FFF7FFFu);
+        m = __vmaxu2(m, v.w & 0x7FFF7FFFu);
+    } else {
+        m = max(m, v.x & 0x7FFFFFFFu);
+        m = max(m, v.y & 0x7FFFFFFFu);
+        m = max(m, v.z & 0x7FFFFFFFu);
+        m = max(m, v.w & 0x7FFFFFFFu);
+    }
+    return m;
+}
+
+// Running maximum -> binary32 magnitude pattern with NaN made canonical.
+template <int WIDE>
+__device__ __forceinline__ uint32_t finish_abs_max(uint32_t m) {
+    if (WIDE == kWideBF16) m = max(m & 0xFFFFu, m >> 16) << 16;
+    return canonical_nan_bits(m);
+}
+
+template <int WIDE>
+__device__ __forceinline__ uint32_t scalar_abs_bits(const void* x, size_t i) {
+    if (WIDE == kWideBF16) return ((uint32_t)(reinterpret_cast<const uint16_t*>(x)[i]) & 0x7FFFu) << 16;
+    return reinterpret_cast<const uint32_t*>(x)[i] & 0x7FFFFFFFu;
+}
+
+template <int WIDE>
+__device__ __forceinline__ float scalar_load(const void* x, size_t i) {
+    if (WIDE == kWideBF16) return __uint_as_float((uint32_t)(reinterpret_cast<const uint16_t*>(x)[i]) << 16);
+    return reinterpret_cast<const float*>(x)[i];
+}
+
+// True when the hardware convert cannot be used for this group of scaled values:
+// a NaN or infinity is present (y * 0 is NaN exactly then), or, in the
+// non-saturating mode, a magnitude reaches the overflow threshold.
+template <int FMT, bool NOSAT, int N>
+__device__ __forceinline__ bool needs_scalar_path(const float (&y)[N]) {
+    float poison = 0.0f;
+#pragma unroll
+    for (int i = 0; i < N; ++i) poison = fmaf(y[i], 0.0f, poison);
+    bool slow = poison != poison;
+    if (NOSAT) {
+        float top = 0.0f;
+#pragma unroll
+        for (int i = 0; i < N; ++i) top = fmaxf(top, fabsf(y[i]));
+        slow = slow || (Fmt<FMT>::nosat_limit_inclusive ? top >= Fmt<FMT>::nosat_limit : top > Fmt<FMT>::nosat_limit);
+    }
+    return slow;
+}
+
+// 8 bf16 values (one 16-byte item) -> 8 codes.
+template <int FMT, bool NOSAT>
+__device__ __forceinline__ uint2 quantize_item_bf16(const uint4& v, float scale) {
+    float y[8];
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        y[2 * i] = __uint_as_float(w[i] << 16) * scale;
+        y[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u) * scale;
+    }
+    uint2 c;
+    if (!needs_scalar_path<FMT, NOSAT>(y)) {
+        c.x = cvt_quad<FMT>(y[0], y[1], y[2], y[3]);
+        c.y = cvt_quad<FMT>(y[4], y[5], y[6], y[7]);
+    } else {
+        c.x = encode_scalar<FMT, NOSAT>(y[0]) | (encode_scalar<FMT, NOSAT>(y[1]) << 8) |
+              (encode_scalar<FMT, NOSAT>(y[2]) << 16) | (encode_scalar<FMT, NOSAT>(y[3]) << 24);
+        c.y = encode_scalar<FMT, NOSAT>(y[4]) | (encode_scalar<FMT, NOSAT>(y[5]) << 8) |
+              (encode_scalar<FMT, NOSAT>(y[6]) << 16) | (encode_scalar<FMT, NOSAT>(y[7]) << 24);
+    }
+    return c;
+}
+
+// 4 binary32 values (one 16-byte item) -> 4 codes.
+template <int FMT, bool NOSAT>
+__device__ __forceinline__ uint32_t quantize_item_f32(const uint4& v, float scale) {
+    float y[4] = {__uint_as_float(v.x) * scale, __uint_as_float(v.y) * scale,
+                  __uint_as_float(v.z) * scale, __uint_as_float(v.w) * scale};
+    if (!needs_scalar_path<FMT, NOSAT>(y)) return cvt_quad<FMT>(y[0], y[1], y[2], y[3]);
+    return encode_scalar<FMT, NOSAT>(y[0]) | (encode_scalar<FMT, NOSAT>(y[1]) << 8) |
+           (encode_scalar<FMT, NOSAT>(y[2]) << 16) | (encode_scalar<FMT, NOSAT>(y[3]) << 24);
+}
+
+// ---------------------------------------------------------------------------
+// kernels: 16-byte aligned fast path
+// ---------------------------------------------------------------------------
+
+// amax over n elements; *amax_bits must be zero before the launch.
+template <int WIDE, int UNROLL>
+__global__ void __launch_bounds__(kThreads) k_amax(const void* __restrict__ x, size_t n, uint32_t* amax_bits) {
+    __shared__ uint32_t red[32];
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;              // elements per 16-byte item
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    const size_t n_items = n / EPI;
+    const size_t per_chunk = (size_t)kThreads * UNROLL;
+    const size_t n_chunks = (n_items + per_chunk - 1) / per_chunk;
+    uint32_t m = 0;
+    for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        const size_t base = chunk * per_chunk + threadIdx.x;
+        uint4 v[UNROLL];
+        if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) m = fold_abs_max<WIDE>(m, v[u]);
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const size_t i = base + (size_t)u * kThreads;
+                if (i < n_items) m = fold_abs_max<WIDE>(m, ld_nc_v4(xv + i));
+            }
+        }
+    }
+    m = finish_abs_max<WIDE>(m);
+    if (blockIdx.x == 0 && threadIdx.x < n - n_items * EPI)      // ragged tail, fewer than EPI elements
+        m = max(m, canonical_nan_bits(scalar_abs_bits<WIDE>(x, n_items * EPI + threadIdx.x)));
+    block_atomic_max_bits(m, red, amax_bits);
+}
+
+// quantize n elements (+ optional amax of the input in the same pass).
+template <int WIDE, int FMT, bool NOSAT, bool WITH_AMAX, int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale_dev,
+           uint8_t* __restrict__ out, uint32_t* amax_bits) {
+    __shared__ uint32_t red[32];
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    const float scale = *scale_dev;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    const size_t n_items = n / EPI;
+    const size_t per_chunk = (size_t)kThreads * UNROLL;
+    const size_t n_chunks = (n_items + per_chunk - 1) / per_chunk;
+    uint32_t m = 0;
+
+    auto emit = [&](size_t i, const uint4& v) {
+        if (WITH_AMAX) m = fold_abs_max<WIDE>(m, v);
+        if (WIDE == kWideBF16) reinterpret_cast<uint2*>(out)[i] = quantize_item_bf16<FMT, NOSAT>(v, scale);
+        else                   reinterpret_cast<uint32_t*>(out)[i] = quantize_item_f32<FMT, NOSAT>(v, scale);
+    };
+
+    for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        const size_t base = chunk * per_chunk + threadIdx.x;
+        if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
+            uint4 v[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) emit(base + (size_t)u * kThreads, v[u]);
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const size_t i = base + (size_t)u * kThreads;
+                if (i < n_items) emit(i, ld_nc_v4(xv + i));
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < n - n_items * EPI) {    // ragged tail
+        const size_t i = n_items * EPI + threadIdx.x;
+        if (WITH_AMAX) {
+            const uint32_t b = scalar_abs_bits<WIDE>(x, i);
+            m = WIDE == kWideBF16 ? __vmaxu2(m, b >> 16) : max(m, b);    // bf16 keeps two packed 16-bit lanes
+        }
+        out[i] = (uint8_t)encode_scalar<FMT, NOSAT>(scalar_load<WIDE>(x, i) * scale);
+    }
+    if (WITH_AMAX) block_atomic_max_bits(finish_abs_max<WIDE>(m), red, amax_bits);
+}
+
+// dequantize: 8 codes (bf16 out) or 4 codes (f32 out) per item, one 16-byte store each.
+template <int FMT, int WIDE, int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+k_dequantize(const uint8_t* __restrict__ c, size_t n, const float* __restrict__ scale_inv_dev, void* __restrict__ out) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    const float si = *scale_inv_dev;
+    const size_t n_items = n / EPI;
+    const size_t per_chunk = (size_t)kThreads * UNROLL;
+    const size_t n_chunks = (n_items + per_chunk - 1) / per_chunk;
+
+    auto emit_bf16 = [&](size_t i, uint2 w) {
+        const float2 a = decode_pair<FMT>(w.x), b = decode_pair<FMT>(w.x >> 16);
+        const float2 d = decode_pair<FMT>(w.y), e = decode_pair<FMT>(w.y >> 16);
+        uint4 o;
+        o.x = pack_bf16(a.x * si, a.y * si);
+        o.y = pack_bf16(b.x * si, b.y * si);
+        o.z = pack_bf16(d.x * si, d.y * si);
+        o.w = pack_bf16(e.x * si, e.y * si);
+        reinterpret_cast<uint4*>(out)[i] = o;
+    };
+    auto emit_f32 = [&](size_t i, uint32_t w) {
+        const float2 a = decode_pair<FMT>(w), b = decode_pair<FMT>(w >> 16);
+        reinterpret_cast<float4*>(out)[i] = make_float4(a.x * si, a.y * si, b.x * si, b.y * si);
+    };
+
+    for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        const size_t base = chunk * per_chunk + threadIdx.x;
+        const bool full = base + (size_t)(UNROLL - 1) * kThreads < n_items;
+        if (WIDE == kWideBF16) {
+            uint2 v[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const size_t i = base + (size_t)u * kThreads;
+                if (full || i < n_items) v[u] = ld_nc_v2(c + i * 8);
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const size_t i = base + (size_t)u * kThreads;
+                if (full || i < n_items) emit_bf16(i, v[u]);
+            }
+        } else {
+            uint32_t v[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const size_t i = base + (size_t)u * kThreads;
+                if (full || i < n_items) v[u] = ld_nc_u32(c + i * 4);
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const size_t i = base + (size_t)u * kThreads;
+                if (full || i < n_items) emit_f32(i, v[u]);
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < n - n_items * EPI) {    // ragged tail
+        const size_t i = n_items * EPI + threadIdx.x;
+        const float v = decode_pair<FMT>(c[i]).x * si;
+        if (WIDE == kWideBF16) reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)pack_bf16(v, 0.0f);
+        else                   reinterpret_cast<float*>(out)[i] = v;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// kernels: element-wise path for pointers that are not 16-byte aligned
+// ---------------------------------------------------------------------------
+
+template <int WIDE>
+__global__ void __launch_bounds__(kThreads) k_amax_elementwise(const void* __restrict__ x, size_t n, uint32_t* amax_bits) {
+    __shared__ uint32_t red[32];
+    uint32_t m = 0;
+    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (size_t)gridDim.x * kThreads)
+        m = max(m, scalar_abs_bits<WIDE>(x, i));
+    block_atomic_max_bits(canonical_nan_bits(m), red, amax_bits);
+}
+
+template <int WIDE, int FMT, bool NOSAT, bool WITH_AMAX>
+__global__ void __launch_bounds__(kThreads)
+k_quantize_elementwise(const void* __restrict__ x, size_t n, const float* __restrict__ scale_dev,
+                       uint8_t* __restrict__ out, uint32_t* amax_bits) {
+    __shared__ uint32_t red[32];
+    const float scale = *scale_dev;
+    uint32_t m = 0;
+    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (size_t)gridDim.x * kThreads) {
+        if (WITH_AMAX) m = max(m, scalar_abs_bits<WIDE>(x, i));
+        out[i] = (uint8_t)encode_scalar<FMT, NOSAT>(scalar_load<WIDE>(x, i) * scale);
+    }
+    if (WITH_AMAX) block_atomic_max_bits(canonical_nan_bits(m), red, amax_bits);
+}
+
+template <int FMT, int WIDE>
+__global__ void __launch_bounds__(kThreads)
+k_dequantize_elementwise(const uint8_t* __restrict__ c, size_t n, const float* __restrict__ scale_inv_dev, void* __restrict__ out) {
+    const float si = *scale_inv_dev;
+    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (size_t)gridDim.x * kThreads) {
+        const float v = decode_pair<FMT>(c[i]).x * si;
+        if (WIDE == kWideBF16) reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)pack_bf16(v, 0.0f);
+        else                   reinterpret_cast<float*>(out)[i] = v;
+    }
+}
+
+// scale = fmax / amax with the guards of the interface; one thread.
+__global__ void k_scale_from_amax(const float* amax_dev, float fmax, float* scale_dev, float* scale_inv_dev) {
+    const float a = *amax_dev;
+    float s = 1.0f;
+    if (a == a && a != 0.0f && fabsf(a) != __int_as_float(0x7F800000)) {
+        s = __fdiv_rn(fmax, a);
+        if (fabsf(s) == __int_as_float(0x7F800000)) s = __int_as_float(0x7F7FFFFF);
+    }
+    *scale_dev = s;
+    *scale_inv_dev = __fdiv_rn(1.0f, s);
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Persistent grid: enough blocks to fill every SM, no more than there is work.
+template <typename Kernel>
+static int persistent_grid(Kernel kernel, size_t work_chunks) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    size_t g = (size_t)sm_count() * (size_t)per_sm;
+    if (g > work_chunks) g = work_chunks;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+static size_t chunks_of(size_t n, int epi, int unroll) {
+    const size_t items = n / (size_t)epi;
+    const size_t per_chunk = (size_t)kThreads * (size_t)unroll;
+    return (items + per_chunk - 1) / per_chunk;
+}
+
+constexpr int kAmaxUnroll = 8;
+constexpr int kQuantUnrollBF16 = 4;
+constexpr int kQuantUnrollF32 = 8;
+constexpr int kDequantUnroll = 4;
+
+template <int WIDE>
+static fp8_status launch_amax(const void* x, size_t n, uint32_t* bits, cudaStream_t st) {
+    if (aligned16(x)) {
+        auto k = k_amax<WIDE, kAmaxUnroll>;
+        const int grid = persistent_grid(k, chunks_of(n, WIDE == kWideBF16 ? 8 : 4, kAmaxUnroll));
+        k<<<grid, kThreads, 0, st>>>(x, n, bits);
+    } else {
+        auto k = k_amax_elementwise<WIDE>;
+        const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
+        k<<<grid, kThreads, 0, st>>>(x, n, bits);
+    }
+    count_launches(1);
+    return launch_status();
+}
+
+template <int WIDE, int FMT, bool NOSAT, bool WITH_AMAX>
+static fp8_status launch_quantize(const void* x, size_t n, const float* scale, uint8_t* out, uint32_t* bits, cudaStream_t st) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int UNROLL = WIDE == kWideBF16 ? kQuantUnrollBF16 : kQuantUnrollF32;
+    // the vector path stores EPI codes per item: out must be EPI-byte aligned, x 16-byte aligned
+    if (aligned16(x) && (reinterpret_cast<uintptr_t>(out) & (EPI - 1)) == 0) {
+        auto k = k_quantize<WIDE, FMT, NOSAT, WITH_AMAX, UNROLL>;
+        const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL));
+        k<<<grid, kThreads, 0, st>>>(x, n, scale, out, bits);
+    } else {
+        auto k = k_quantize_elementwise<WIDE, FMT, NOSAT, WITH_AMAX>;
+        const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
+        k<<<grid, kThreads, 0, st>>>(x, n, scale, out, bits);
+    }
+    count_launches(1);
+    return launch_status();
+}
+
+template <int WIDE, int FMT>
+static fp8_status dispatch_quantize(const void* x, size_t n, bool nosat, const float* scale, uint8_t* out, uint32_t* bits, cudaStream_t st) {
+    if (nosat) return bits ? launch_quantize<WIDE, FMT, true, true>(x, n, scale, out, bits, st)
+                           : launch_quantize<WIDE, FMT, true, false>(x, n, scale, out, bits, st);
+    return bits ? launch_quantize<WIDE, FMT, false, true>(x, n, scale, out, bits, st)
+                : launch_quantize<WIDE, FMT, false, false>(x, n, scale, out, bits, st);
+}
+
+template <int FMT, int WIDE>
+static fp8_status launch_dequantize(const uint8_t* c, size_t n, const float* si, void* out, cudaStream_t st) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    if (aligned16(out) && (reinterpret_cast<uintptr_t>(c) & (EPI - 1)) == 0) {
+        auto k = k_dequantize<FMT, WIDE, kDequantUnroll>;
+        const int grid = persistent_grid(k, chunks_of(n, EPI, kDequantUnroll));
+        k<<<grid, kThreads, 0, st>>>(c, n, si, out);
+    } else {
+        auto k = k_dequantize_elementwise<FMT, WIDE>;
+        const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
+        k<<<grid, kThreads, 0, st>>>(c, n, si, out);
+    }
+    count_launches(1);
+    return launch_status();
+}
+
+static fp8_status zero_word(void* p, cudaStream_t st) {
+    if (cudaMemsetAsync(p, 0, 4, st) != cudaSuccess) return FP8_ERR_CUDA;
+    count_launches(1);
+    return FP8_OK;
+}
+
+}  // namespace fp8b200
+
+using namespace fp8b200;
+
+extern "C" {
+
+fp8_status fp8_amax(const void* x, fp8_wide t, size_t n, float* amax_dev, void* stream) {
+    if (!amax_dev || (!x && n)) return FP8_ERR_NULL;
+    if (t != FP8_F32 && t != FP8_BF16) return FP8_ERR_ENUM;
+    cudaStream_t st = (cudaStream_t)stream;
+    fp8_status s = zero_word(amax_dev, st);
+    if (s != FP8_OK || n == 0) return s;
+    uint32_t* bits = reinterpret_cast<uint32_t*>(amax_dev);
+    return t == FP8_F32 ? launch_amax<kWideF32>(x, n, bits, st) : launch_amax<kWideBF16>(x, n, bits, st);
+}
+
+fp8_status fp8_scale_from_amax(const float* amax_dev, fp8_format f, float* scale_dev, float* scale_inv_dev, void* stream) {
+    if (!amax_dev || !scale_dev || !scale_inv_dev) return FP8_ERR_NULL;
+    if (f != FP8_E4M3 && f != FP8_E5M2) return FP8_ERR_ENUM;
+    k_scale_from_amax<<<1, 1, 0, (cudaStream_t)stream>>>(amax_dev, f == FP8_E4M3 ? 448.0f : 57344.0f, scale_dev, scale_inv_dev);
+    count_launches(1);
+    return launch_status();
+}
+
+fp8_status fp8_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o,
+                        const float* scale_dev, uint8_t* out, float* amax_dev, void* stream) {
+    if (!scale_dev || ((!x || !out) && n)) return FP8_ERR_NULL;
+    if ((t != FP8_F32 && t != FP8_BF16) || (f != FP8_E4M3 && f != FP8_E5M2) || (o != FP8_SATURATE && o != FP8_NOSAT))
+        return FP8_ERR_ENUM;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (amax_dev) {
+        fp8_status s = zero_word(amax_dev, st);
+        if (s != FP8_OK) return s;
+    }
+    if (n == 0) return FP8_OK;
+    uint32_t* bits = reinterpret_cast<uint32_t*>(amax_dev);
+    const bool nosat = o == FP8_NOSAT;
+    if (t == FP8_F32)
+        return f == FP8_E4M3 ? dispatch_quantize<kWideF32, kE4M3>(x, n, nosat, scale_dev, out, bits, st)
+                             : dispatch_quantize<kWideF32, kE5M2>(x, n, nosat, scale_dev, out, bits, st);
+    return f == FP8_E4M3 ? dispatch_quantize<kWideBF16, kE4M3>(x, n, nosat, scale_dev, out, bits, st)
+                         : dispatch_quantize<kWideBF16, kE5M2>(x, n, nosat, scale_dev, out, bits, st);
+}
+
+fp8_status fp8_dequantize(const uint8_t* c, size_t n, fp8_format f, const float* scale_inv_dev, void* out, fp8_wide t, void* stream) {
+    if (!scale_inv_dev || ((!c || !out) && n)) return FP8_ERR_NULL;
+    if ((t != FP8_F32 && t != FP8_BF16) || (f != FP8_E4M3 && f != FP8_E5M2)) return FP8_ERR_ENUM;
+    if (n == 0) return FP8_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (t == FP8_F32)
+        return f == FP8_E4M3 ? launch_dequantize<kE4M3, kWideF32>(c, n, scale_inv_dev, out, st)
+                             : launch_dequantize<kE5M2, kWideF32>(c, n, scale_inv_dev, out, st);
+    return f == FP8_E4M3 ? launch_dequantize<kE4M3, kWideBF16>(c, n, scale_inv_dev, out, st)
+                         : launch_dequantize<kE5M2, kWideBF16>(c, n, scale_inv_dev, out, st);
+}
+
+const char* fp8_status_string(fp8_status s) {
+    switch (s) {
+        case FP8_OK: return "ok";
+        case FP8_ERR_NULL: return "null pointer";
+        case FP8_ERR_ENUM: return "enum out of range";
+        case FP8_ERR_SHAPE: return "bad shape or leading dimension";
+        case FP8_ERR_ALIGN: return "operand not 16-byte aligned";
+        case FP8_ERR_UNSUPPORTED: return "unsupported size";
+        case FP8_ERR_CUDA: return "CUDA error";
+        case FP8_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+uint64_t fp8_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,507 @@
+// FP8 GEMM on the 5th-generation tensor cores (sm_100a): Sections 2 and 4.1 of
+// the paper: dot products of FP8 inputs accumulated in binary32, unscaled once
+// per dot product, written in a wider type.
+//
+// One persistent CTA per SM works through 128 x 256 output tiles.
+//   warp 0       TMA producer: cp.async.bulk.tensor loads of A (128 x 128 B) and
+//                B (256 x 128 B) K-blocks into a 4-stage 128B-swizzled smem ring
+//   warp 1       TMEM allocation, and one elected lane issuing tcgen05.mma
+//                (kind::f8f6f4, M128 N256 K32) into one of two 256-column TMEM
+//                accumulators; tcgen05.commit releases smem stages / publishes
+//                the finished accumulator
+//   warps 2..5   epilogue: tcgen05.ld of the accumulator (each warp owns its 32
+//                TMEM lanes), multiply by sa_inv*sb_inv, round to bf16 / keep
+//                fp32, amax of the stored values, global stores.  The epilogue
+//                of tile i overlaps the main loop of tile i+1.
+// Operands may be K-major or MN-major (forward / dgrad / wgrad layouts); the
+// two formats of a mixed E5M2 x E4M3 product are set in the instruction
+// descriptor.  No TMA multicast is used anywhere.
+// Every mbarrier wait is bounded: on expiry the kernel latches an error code,
+// all roles drain, TMEM is freed and the kernel returns.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <mutex>
+
+#include "codec.cuh"
+#include "common.cuh"
+
+namespace fp8b200 {
+
+__device__ unsigned int g_async_latch[2] = {0u, 0u};
+
+namespace gemm {
+
+constexpr int BM = 128;             // tile rows  (= UMMA M, one TMEM lane per row)
+constexpr int BN = 256;             // tile cols  (= UMMA N, one TMEM column per col)
+constexpr int BK = 128;             // K-block in elements = bytes = one 128B swizzle row
+constexpr int UMMA_K = 32;          // K of one tcgen05.mma for 8-bit operands
+constexpr int STAGES = 4;
+constexpr int ACC_STAGES = 2;       // 2 x 256 columns = all 512 TMEM columns
+constexpr int THREADS = 192;
+constexpr int EPI_WARPS = 4;
+constexpr uint32_t A_BYTES = BM * BK;          // 16 KiB
+constexpr uint32_t B_BYTES = BN * BK;          // 32 KiB
+constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t SMEM_TILES = STAGES * STAGE_BYTES;
+constexpr uint32_t SMEM_BARRIERS = 256;
+constexpr uint32_t SMEM_BYTES = SMEM_TILES + SMEM_BARRIERS + 1024;   // + slack to align the ring to 1024 B
+constexpr uint32_t TMEM_COLS = 512;
+constexpr int GROUP_M = 8;          // tile raster: GROUP_M row-tiles share each sweep over N
+
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
+
+// codes written to the error latch
+enum : uint32_t { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC_EMPTY = 3, WAIT_ACC_FULL = 4 };
+
+// ---- PTX wrappers ----------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false after WAIT_LIMIT_NS, or at once when another
+// role has already given up (abort flag), having latched `code`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1u;
+                if (atomicCAS(&g_async_latch[0], 0u, code) == 0u) g_async_latch[1] = blockIdx.x;
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_f8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading and
+// stride byte offsets in 16-byte units, version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;          // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;          // SWIZZLE_128B
+    return d;
+}
+
+struct Params {
+    int64_t M, N, K;
+    int64_t ldd;                    // elements
+    void* D;
+    const float* sa_inv;
+    const float* sb_inv;
+    uint32_t* amax_bits;            // may be null
+    uint32_t idesc;
+    int tiles_m, tiles_n;
+};
+
+struct alignas(8) Barriers {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t acc_full[ACC_STAGES];
+    uint64_t acc_empty[ACC_STAGES];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+static_assert(sizeof(Barriers) <= SMEM_BARRIERS, "barrier block too large");
+
+// tile index -> (row-tile, col-tile): GROUP_M row-tiles advance together over N,
+// so that the CTAs running at one time share their A and B panels in L2.
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tm, int& tn) {
+    const int per_group = GROUP_M * tiles_n;
+    const int g = t / per_group;
+    const int first_m = g * GROUP_M;
+    const int rows = min(GROUP_M, tiles_m - first_m);
+    const int r = t - g * per_group;
+    tm = first_m + r % rows;
+    tn = r / rows;
+}
+
+// A_MN / B_MN: operand stored with its M (resp. N) index contiguous.
+// OUT_BF16: D is bf16, else fp32.
+template <bool A_MN, bool B_MN, bool OUT_BF16>
+__global__ void __launch_bounds__(THREADS, 1)
+k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t ring = (raw + 1023u) & ~1023u;                 // 1024-byte aligned tile ring
+    Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (ring - raw) + SMEM_TILES);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int k_blocks = (int)((p.K + BK - 1) / BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
+        for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(smem_u32(&bars->acc_full[a]), 1); mbar_init(smem_u32(&bars->acc_empty[a]), EPI_WARPS); }
+        bars->abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {                                              // whole warp: allocate all 512 TMEM columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            int tm, tn;
+            tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
+            const int m0 = tm * BM, n0 = tn * BN;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, WAIT_EMPTY);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t full = smem_u32(&bars->full[stage]);
+                    const uint32_t sa = ring + stage * STAGE_BYTES;
+                    const uint32_t sb = sa + A_BYTES;
+                    const int k0 = kb * BK;
+                    mbar_arrive_expect_tx(full, STAGE_BYTES);
+                    if (A_MN) tma_load_2d(sa, &map_a, m0, k0, full);          // box {128 m, 128 k}
+                    else      tma_load_2d(sa, &map_a, k0, m0, full);          // box {128 k, 128 m}
+                    if (B_MN) {                                               // two boxes {128 n, 128 k}
+                        tma_load_2d(sb, &map_b, n0, k0, full);
+                        tma_load_2d(sb + B_BYTES / 2, &map_b, n0 + 128, k0, full);
+                    } else {
+                        tma_load_2d(sb, &map_b, k0, n0, full);                // box {128 k, 256 n}
+                    }
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        int it = 0;
+        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+            const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
+            ok = mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag, WAIT_ACC_EMPTY);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t tmem_d = tmem_base + acc * BN;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, WAIT_FULL);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t sa = ring + stage * STAGE_BYTES;
+                    const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // K-major: 8-row groups 1024 B apart, +32 B per K step inside the swizzled row.
+                        // MN-major: 8-k groups 1024 B apart, 128-wide MN blocks BK*128 B apart, +32 k-rows per step.
+                        const uint64_t da = A_MN ? smem_desc(sa + k * UMMA_K * 128, BK * 128, 1024)
+                                                 : smem_desc(sa + k * UMMA_K, 16, 1024);
+                        const uint64_t db = B_MN ? smem_desc(sb + k * UMMA_K * 128, BK * 128, 1024)
+                                                 : smem_desc(sb + k * UMMA_K, 16, 1024);
+                        tc_mma_f8(tmem_d, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&bars->empty[stage]));                 // frees the smem stage when the MMAs retire
+                    if (kb == k_blocks - 1) tc_commit(smem_u32(&bars->acc_full[acc]));
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;                                   // TMEM lane quarter this warp may read
+        const float alpha = __ldg(p.sa_inv) * __ldg(p.sb_inv);
+        uint32_t running = 0;                                     // max of stored magnitude bits (bf16: 16-bit patterns)
+        bool ok = true;
+        int it = 0;
+        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+            int tm, tn;
+            tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
+            const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
+            ok = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, WAIT_ACC_FULL);
+            if (!ok) break;
+            tc_fence_after();
+            const int64_t row = (int64_t)tm * BM + q * 32 + lane;
+            const int64_t col0 = (int64_t)tn * BN;
+            const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tc_ld32(taddr + c * 32, r);
+                tc_wait_ld();
+                const int64_t col = col0 + c * 32;
+                if (row < p.M && col < p.N) {
+                    const bool full_chunk = col + 32 <= p.N;
+                    if (OUT_BF16) {
+                        uint16_t* dst = reinterpret_cast<uint16_t*>(p.D) + row * p.ldd + col;
+                        uint32_t w[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            w[i] = pack_bf16(__uint_as_float(r[2 * i]) * alpha, __uint_as_float(r[2 * i + 1]) * alpha);
+                        }
+                        if (full_chunk) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) running = __vmaxu2(running, w[i] & 0x7FFF7FFFu);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+                        } else {
+                            for (int i = 0; i < 32 && col + i < p.N; ++i) {
+                                const uint32_t h = (i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu);
+                                running = __vmaxu2(running, h & 0x7FFFu);
+                                dst[i] = (uint16_t)h;
+                            }
+                        }
+                    } else {
+                        float* dst = reinterpret_cast<float*>(p.D) + row * p.ldd + col;
+                        if (full_chunk) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                float4 v;
+                                v.x = __uint_as_float(r[4 * i]) * alpha;
+                                v.y = __uint_as_float(r[4 * i + 1]) * alpha;
+                                v.z = __uint_as_float(r[4 * i + 2]) * alpha;
+                                v.w = __uint_as_float(r[4 * i + 3]) * alpha;
+                                running = max(running, max(max(__float_as_uint(v.x) & 0x7FFFFFFFu, __float_as_uint(v.y) & 0x7FFFFFFFu),
+                                                           max(__float_as_uint(v.z) & 0x7FFFFFFFu, __float_as_uint(v.w) & 0x7FFFFFFFu)));
+                                reinterpret_cast<float4*>(dst)[i] = v;
+                            }
+                        } else {
+                            for (int i = 0; i < 32 && col + i < p.N; ++i) {
+                                const float v = __uint_as_float(r[i]) * alpha;
+                                running = max(running, __float_as_uint(v) & 0x7FFFFFFFu);
+                                dst[i] = v;
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[acc]));      // accumulator may be overwritten
+        }
+        if (p.amax_bits) {
+            uint32_t bits = OUT_BF16 ? (max(running & 0xFFFFu, running >> 16) << 16) : running;
+            bits = warp_max_u32(canonical_nan_bits(bits));
+            if (lane == 0 && bits != 0u) atomicMax(p.amax_bits, bits);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// K == 0: D = 0.
+template <bool OUT_BF16>
+__global__ void k_zero_d(void* D, int64_t M, int64_t N, int64_t ldd) {
+    const int64_t total = M * N;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / N, c = i - r * N;
+        if (OUT_BF16) reinterpret_cast<uint16_t*>(D)[r * ldd + c] = 0;
+        else          reinterpret_cast<float*>(D)[r * ldd + c] = 0.0f;
+    }
+}
+
+// ---- host ------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    });
+    return fn;
+}
+
+// 2-D byte tensor {inner, outer} with row pitch `pitch`, box {box_inner, box_outer}, 128B swizzle, zero fill.
+static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch,
+                     uint32_t box_inner, uint32_t box_outer) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {pitch};
+    const cuuint32_t box[2] = {box_inner, box_outer};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool A_MN, bool B_MN, bool OUT_BF16>
+static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid, cudaStream_t st) {
+    auto k = k_gemm_fp8<A_MN, B_MN, OUT_BF16>;
+    // per device and cheap, so set on every launch rather than cached
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return FP8_ERR_CUDA;
+    k<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, p);
+    count_launches(1);
+    return launch_status();
+}
+
+}  // namespace gemm
+}  // namespace fp8b200
+
+using namespace fp8b200;
+
+extern "C" {
+
+fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,
+                    const float* scale_inv_a_dev, const float* scale_inv_b_dev, float* amax_d_dev, void* stream) {
+    using namespace fp8b200::gemm;
+    if (!d || !scale_inv_a_dev || !scale_inv_b_dev) return FP8_ERR_NULL;
+    if ((d->fa != FP8_E4M3 && d->fa != FP8_E5M2) || (d->fb != FP8_E4M3 && d->fb != FP8_E5M2) ||
+        (d->ma != FP8_MAJOR_K && d->ma != FP8_MAJOR_MN) || (d->mb != FP8_MAJOR_K && d->mb != FP8_MAJOR_MN) ||
+        (d->out != FP8_F32 && d->out != FP8_BF16))
+        return FP8_ERR_ENUM;
+    const int64_t M = d->M, N = d->N, K = d->K;
+    if (M < 0 || N < 0 || K < 0) return FP8_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool a_mn = d->ma == FP8_MAJOR_MN, b_mn = d->mb == FP8_MAJOR_MN;
+    const int64_t esz = d->out == FP8_BF16 ? 2 : 4;
+    const int64_t tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
+    // ---- validation: nothing is enqueued before every check has passed
+    if (M > 0 && N > 0) {
+        if (!D) return FP8_ERR_NULL;
+        if (d->ldd < N) return FP8_ERR_SHAPE;
+        if (K > 0) {
+            if (!A || !B) return FP8_ERR_NULL;
+            if (d->lda < (a_mn ? M : K) || d->ldb < (b_mn ? N : K)) return FP8_ERR_SHAPE;
+            if ((reinterpret_cast<uintptr_t>(A) & 15u) || (reinterpret_cast<uintptr_t>(B) & 15u) || (d->lda & 15) || (d->ldb & 15))
+                return FP8_ERR_ALIGN;
+        }
+        if ((reinterpret_cast<uintptr_t>(D) & 15u) || ((d->ldd * esz) & 15)) return FP8_ERR_ALIGN;
+        if (tiles_m * tiles_n > (int64_t)1 << 30 || M > ((int64_t)1 << 31) - 256 || N > ((int64_t)1 << 31) - 512 ||
+            K > ((int64_t)1 << 31) - 256)
+            return FP8_ERR_UNSUPPORTED;
+    }
+    // ---- work
+    if (amax_d_dev) {
+        if (cudaMemsetAsync(amax_d_dev, 0, 4, st) != cudaSuccess) return FP8_ERR_CUDA;
+        count_launches(1);
+    }
+    if (M == 0 || N == 0) return FP8_OK;
+    if (K == 0) {
+        const int grid = sm_count() * 4;
+        if (d->out == FP8_BF16) k_zero_d<true><<<grid, 256, 0, st>>>(D, M, N, d->ldd);
+        else                    k_zero_d<false><<<grid, 256, 0, st>>>(D, M, N, d->ldd);
+        count_launches(1);
+        return launch_status();
+    }
+
+    CUtensorMap map_a, map_b;
+    bool ok = a_mn ? make_map(&map_a, A, (uint64_t)M, (uint64_t)K, (uint64_t)d->lda, 128, BK)
+                   : make_map(&map_a, A, (uint64_t)K, (uint64_t)M, (uint64_t)d->lda, BK, BM);
+    ok = ok && (b_mn ? make_map(&map_b, B, (uint64_t)N, (uint64_t)K, (uint64_t)d->ldb, 128, BK)
+                     : make_map(&map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)d->ldb, BK, BN));
+    if (!ok) return FP8_ERR_CUDA;
+
+    Params p;
+    p.M = M; p.N = N; p.K = K; p.ldd = d->ldd; p.D = D;
+    p.sa_inv = scale_inv_a_dev; p.sb_inv = scale_inv_b_dev;
+    p.amax_bits = reinterpret_cast<uint32_t*>(amax_d_dev);
+    p.tiles_m = (int)tiles_m; p.tiles_n = (int)tiles_n;
+    // instruction descriptor: fp32 accumulate, operand formats and majors, N/8, M/16
+    p.idesc = (1u << 4) | ((uint32_t)d->fa << 7) | ((uint32_t)d->fb << 10) | ((a_mn ? 1u : 0u) << 15) |
+              ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    int grid = sm_count();
+    if ((int64_t)grid > tiles_m * tiles_n) grid = (int)(tiles_m * tiles_n);
+    const bool bf = d->out == FP8_BF16;
+    if (!a_mn && !b_mn) return bf ? launch<false, false, true>(map_a, map_b, p, grid, st) : launch<false, false, false>(map_a, map_b, p, grid, st);
+    if (!a_mn && b_mn)  return bf ? launch<false, true, true>(map_a, map_b, p, grid, st)  : launch<false, true, false>(map_a, map_b, p, grid, st);
+    if (a_mn && !b_mn)  return bf ? launch<true, false, true>(map_a, map_b, p, grid, st)  : launch<true, false, false>(map_a, map_b, p, grid, st);
+    return bf ? launch<true, true, true>(map_a, map_b, p, grid, st) : launch<true, true, false>(map_a, map_b, p, grid, st);
+}
+
+fp8_status fp8_async_status(uint32_t* detail) {
+    unsigned int latch[2] = {0u, 0u};
+    if (cudaDeviceSynchronize() != cudaSuccess) return FP8_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(latch, g_async_latch, sizeof(latch)) != cudaSuccess) return FP8_ERR_CUDA;
+    if (detail) *detail = latch[0];
+    if (latch[0] == 0u) return FP8_OK;
+    const unsigned int zero[2] = {0u, 0u};
+    if (cudaMemcpyToSymbol(g_async_latch, zero, sizeof(zero)) != cudaSuccess) return FP8_ERR_CUDA;
+    return FP8_ERR_TIMEOUT;
+}
+
+}  // extern "C"

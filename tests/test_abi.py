@@ -1,0 +1,64 @@
+"""The C-ABI library builds, loads, and exports every entry point the header declares.
+Runs without a GPU: only calls that return before touching the device are made."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2209_05433_b200 import api
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "fp8_b200.h")
+
+
+def _declared():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(fp8_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_and_binding_name_the_same_entry_points():
+    assert _declared() == sorted(api.EXPORTS)
+    for name in ("fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_dequantize", "fp8_gemm"):
+        assert callable(getattr(api, name))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = api.load()
+    for name in _declared():
+        assert hasattr(lib, name), name
+    assert lib.fp8_status_string(0) == b"ok"
+    assert lib.fp8_status_string(4) == b"operand not 16-byte aligned"
+    assert lib.fp8_status_string(99) == b"unknown status"
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    lib = api.load()
+    one = ctypes.c_void_p(16)          # never dereferenced: every call below fails validation first
+    assert lib.fp8_amax(one, 0, 4, None, None) == 1                      # FP8_ERR_NULL
+    assert lib.fp8_amax(one, 7, 4, one, None) == 2                       # FP8_ERR_ENUM
+    assert lib.fp8_scale_from_amax(None, 0, one, one, None) == 1
+    assert lib.fp8_scale_from_amax(one, 5, one, one, None) == 2
+    assert lib.fp8_quantize(one, 1, 4, 0, 0, None, one, None, None) == 1
+    assert lib.fp8_quantize(one, 1, 4, 3, 0, one, one, None, None) == 2
+    assert lib.fp8_quantize(one, 1, 4, 0, 2, one, one, None, None) == 2
+    assert lib.fp8_dequantize(one, 4, 0, None, one, 1, None) == 1
+    assert lib.fp8_dequantize(one, 4, 9, one, one, 1, None) == 2
+    d = api.GemmDesc(128, 128, 128, 0, 0, 0, 0, 128, 128, 128, 1)
+    assert lib.fp8_gemm(None, one, one, one, one, one, None, None) == 1
+    assert lib.fp8_gemm(ctypes.byref(d), one, one, one, None, one, None, None) == 1
+    d.fa = 4
+    assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 2
+    d.fa = 0
+    d.M = -1
+    assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 3       # FP8_ERR_SHAPE
+    d.M = 128
+    d.lda = 64                                                                          # smaller than K
+    assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 3
+    d.lda = 136                                                                         # not a multiple of 16
+    assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 4       # FP8_ERR_ALIGN
+    d.lda = 128
+    assert lib.fp8_gemm(ctypes.byref(d), ctypes.c_void_p(24), one, one, one, one, None, None) == 4
+    d.ldd = 100                                                                         # smaller than N
+    assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 3

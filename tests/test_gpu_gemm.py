@@ -1,0 +1,198 @@
+"""GPU parity of fp8_gemm against the CPU oracle (fp64 accumulation over decoded codes).
+fp32 output: |gpu - ref| <= 1e-5 * sum_k |a.b| per element.  bf16 output: within 1 bf16 ulp of the
+correctly rounded value of some v inside that interval (equal to "1 ulp of the rounded reference"
+whenever the accumulation error is far below one bf16 ulp of the result)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2209_05433_b200 import api, synth
+from tests._util import THREADS, check_gemm_bf16, check_gemm_f32, to_np_bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+E4, E5 = oracle.E4M3, oracle.E5M2
+ROLES = {"fprop": (E4, E4), "dgrad": (E5, E4), "wgrad": (E4, E5)}
+
+
+def _scalar(v):
+    return torch.tensor([v], dtype=torch.float32, device=DEV)
+
+
+def _codes(rng, fmt, shape, spread=6.0):
+    """finite random codes with magnitudes spread over a few binades around 1"""
+    x = rng.standard_normal(shape).astype(np.float32) * np.exp2(rng.uniform(-spread, 2, size=shape)).astype(np.float32)
+    return oracle.quantize(x, 1.0, fmt).reshape(shape)
+
+
+def _pad_cols(a_np, mult=16, fill=0x7F):
+    """copy into a buffer whose row pitch is a multiple of 16 bytes; padding holds NaN codes
+    so that any read outside the logical extent would poison the result"""
+    r, c = a_np.shape
+    pitch = (c + mult - 1) // mult * mult
+    buf = np.full((r, pitch), fill, dtype=np.uint8)
+    buf[:, :c] = a_np
+    return buf
+
+
+def _run(A_np, fa, ma, B_np, fb, mb, M, N, K, out_dtype, sa_inv=0.013, sb_inv=0.5, want_amax=True):
+    """A_np is the stored array ([M,K] or [K,M]); B_np the stored array ([N,K] or [K,N])."""
+    A_buf, B_buf = _pad_cols(A_np), _pad_cols(B_np)
+    A = torch.from_numpy(A_buf).to(DEV)[:, : A_np.shape[1]]
+    B = torch.from_numpy(B_buf).to(DEV)[:, : B_np.shape[1]]
+    esz = 2 if out_dtype == torch.bfloat16 else 4
+    ldd = (N * esz + 15) // 16 * 16 // esz
+    D_full = torch.full((M + 1, ldd), 777.0, dtype=out_dtype, device=DEV)       # guard row and pad columns
+    D = D_full[:M, :N]
+    amax = _scalar(-1.0) if want_amax else None
+    api.fp8_gemm(A, fa, ma, B, fb, mb, D, _scalar(sa_inv), _scalar(sb_inv), amax)
+    torch.cuda.synchronize()
+    st, detail = api.fp8_async_status()
+    assert st == 0, "device-side wait expired, code %d" % detail
+    assert bool((D_full[M:, :] == 777.0).all()) and bool((D_full[:M, N:] == 777.0).all()), "wrote outside D"
+    a_str = (A_buf.shape[1], 1) if ma == api.MAJOR_K else (1, A_buf.shape[1])
+    b_str = (1, B_buf.shape[1]) if mb == api.MAJOR_K else (B_buf.shape[1], 1)
+    ref, sabs = oracle.gemm_rows(A_buf, fa, a_str, B_buf, fb, b_str, N, K, 0, M, sa_inv, sb_inv, threads=THREADS)
+    got = to_np_bits(D)
+    if out_dtype == torch.float32:
+        ok, worst = check_gemm_f32(got, ref, sabs)
+        assert ok.all(), "fp32: %d of %d outside 1e-5*sum|ab| (worst ratio %.3g) at %s" % (
+            (~ok).sum(), ok.size, worst, np.argwhere(~ok)[:4].tolist())
+    else:
+        ok, literal = check_gemm_bf16(got, ref, sabs, oracle.round_bf16_from_f64)
+        assert ok.all(), "bf16: %d of %d fail at %s" % ((~ok).sum(), ok.size, np.argwhere(~ok)[:4].tolist())
+    if want_amax:
+        # epilogue amax is the amax of D as stored: the library's own fp8_amax and the oracle's amax of
+        # the stored values must both reproduce it bit for bit
+        dense = D.contiguous()
+        a2 = _scalar(-1.0)
+        api.fp8_amax(dense, a2)
+        bits = amax.cpu().numpy().view(np.uint32)[0]
+        assert bits == a2.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(to_np_bits(dense).reshape(-1))
+    return got, ref, sabs
+
+
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_config1_tiny_gemm(out_dtype):
+    """fp32 A, B [256x256] N(0,1) with 0.5% x64 outliers, amax-derived scales, E4M3 x E4M3, M=N=K=256"""
+    M = N = K = 256
+    xa = synth.normal_with_scaled_outliers(M * K, 0, synth.A_ID, 0.005, 64.0, device=DEV)
+    xb = synth.normal_with_scaled_outliers(K * N, 0, synth.B_ID, 0.005, 64.0, device=DEV)
+    qa = torch.empty(M * K, dtype=torch.uint8, device=DEV)
+    qb = torch.empty(K * N, dtype=torch.uint8, device=DEV)
+    sinv = []
+    for x, q in ((xa, qa), (xb, qb)):
+        a, s, si = _scalar(0.0), _scalar(0.0), _scalar(0.0)
+        api.fp8_amax(x, a)
+        api.fp8_scale_from_amax(a, api.E4M3, s, si)
+        api.fp8_quantize(x, api.E4M3, s, q)
+        sinv.append(si)
+    # oracle side from the same wide inputs
+    wa = oracle.scale_from_amax(oracle.amax(to_np_bits(xa)), E4)
+    wb = oracle.scale_from_amax(oracle.amax(to_np_bits(xb)), E4)
+    A_np = oracle.quantize(to_np_bits(xa), wa[0], E4).reshape(M, K)
+    B_np = oracle.quantize(to_np_bits(xb), wb[0], E4).reshape(K, N)      # stored [K,N]: N contiguous
+    assert np.array_equal(qa.cpu().numpy().reshape(M, K), A_np) and np.array_equal(qb.cpu().numpy().reshape(K, N), B_np)
+    D = torch.empty(M, N, dtype=out_dtype, device=DEV)
+    api.fp8_gemm(qa.view(M, K), api.E4M3, api.MAJOR_K, qb.view(K, N), api.E4M3, api.MAJOR_MN, D, sinv[0], sinv[1])
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    ref, sabs = oracle.gemm_rows(A_np, E4, (K, 1), B_np, E4, (N, 1), N, K, 0, M, wa[1], wb[1], threads=THREADS)
+    if out_dtype == torch.float32:
+        ok, worst = check_gemm_f32(to_np_bits(D), ref, sabs)
+        assert ok.all(), worst
+    else:
+        ok, literal = check_gemm_bf16(to_np_bits(D), ref, sabs, oracle.round_bf16_from_f64)
+        assert ok.all()
+
+
+@pytest.mark.parametrize("role", list(ROLES))
+@pytest.mark.parametrize("ma", [api.MAJOR_K, api.MAJOR_MN])
+@pytest.mark.parametrize("mb", [api.MAJOR_K, api.MAJOR_MN])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_layouts_formats_and_outputs(role, ma, mb, out_dtype):
+    """several tiles in each direction, several K blocks, every operand layout and format pair"""
+    fa, fb = ROLES[role]
+    M, N, K = 384, 768, 640
+    rng = np.random.default_rng(1000 + list(ROLES).index(role) * 4 + ma * 2 + mb)
+    A_np = _codes(rng, fa, (M, K) if ma == api.MAJOR_K else (K, M))
+    B_np = _codes(rng, fb, (N, K) if mb == api.MAJOR_K else (K, N))
+    _run(A_np, fa, ma, B_np, fb, mb, M, N, K, out_dtype)
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 8, 16), (100, 40, 48), (129, 257, 129), (300, 520, 200), (128, 256, 128),
+                                    (257, 8, 1000), (5, 1000, 33)])
+@pytest.mark.parametrize("ma,mb", [(api.MAJOR_K, api.MAJOR_K), (api.MAJOR_K, api.MAJOR_MN), (api.MAJOR_MN, api.MAJOR_MN)])
+def test_ragged_edges(M, N, K, ma, mb):
+    """sizes that are not multiples of the tile; padding columns of A and B hold NaN codes"""
+    rng = np.random.default_rng(M * 1000003 + N * 1009 + K)
+    A_np = _codes(rng, E5, (M, K) if ma == api.MAJOR_K else (K, M))
+    B_np = _codes(rng, E4, (N, K) if mb == api.MAJOR_K else (K, N))
+    for out_dtype in (torch.float32, torch.bfloat16):
+        _run(A_np, E5, ma, B_np, E4, mb, M, N, K, out_dtype)
+
+
+def test_long_k_accumulation_error():
+    """K as long as the workloads' longest contraction dimension (49152): the binary32 accumulation
+    of the tensor cores must stay inside the tolerance"""
+    rng = np.random.default_rng(77)
+    M, N, K = 128, 256, 49152
+    for fa, fb in ((E4, E4), (E5, E4)):
+        A_np = _codes(rng, fa, (M, K), spread=3.0)
+        B_np = _codes(rng, fb, (N, K), spread=3.0)
+        _run(A_np, fa, api.MAJOR_K, B_np, fb, api.MAJOR_K, M, N, K, torch.float32)
+    # all-positive operands: no cancellation, the sum is as large as sum|ab|
+    A_np = _codes(rng, E4, (M, K), spread=1.0) & 0x7F
+    B_np = _codes(rng, E4, (N, K), spread=1.0) & 0x7F
+    _run(A_np, E4, api.MAJOR_K, B_np, E4, api.MAJOR_K, M, N, K, torch.float32)
+    _run(A_np, E4, api.MAJOR_K, B_np, E4, api.MAJOR_K, M, N, K, torch.bfloat16)
+
+
+def test_many_tiles_persistent_schedule():
+    """more tiles than SMs so that every CTA walks several tiles and both accumulators wrap"""
+    rng = np.random.default_rng(3)
+    M, N, K = 128 * 21, 256 * 15, 256            # 315 tiles
+    A_np = _codes(rng, E4, (M, K))
+    B_np = _codes(rng, E4, (K, N))
+    A = torch.from_numpy(A_np).to(DEV)
+    B = torch.from_numpy(B_np).to(DEV)
+    D = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+    amax = _scalar(0.0)
+    api.fp8_gemm(A, E4, api.MAJOR_K, B, E4, api.MAJOR_MN, D, _scalar(0.25), _scalar(0.125), amax)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    # E4M3 x E4M3 with K=256 and power-of-two scales is exact in binary32: compare with fp64 matmul, rounded once
+    t = oracle.decode_table(E4)
+    ref = (t[A_np] @ t[B_np]) * (0.25 * 0.125)
+    want = oracle.round_bf16_from_f64(ref)
+    assert np.array_equal(to_np_bits(D), want)
+    assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(want.reshape(-1))
+
+
+def test_special_codes_and_degenerate_shapes():
+    rng = np.random.default_rng(5)
+    M, N, K = 128, 256, 256
+    A_np = _codes(rng, E5, (M, K))
+    B_np = _codes(rng, E4, (N, K))
+    A_np[3, 7] = 0x7C          # +Inf
+    A_np[9, 1] = 0xFC          # -Inf
+    A_np[20, 2] = 0x7E         # E5M2 NaN
+    B_np[40, 100] = 0x7F       # E4M3 NaN
+    A_np[50, 5] = 0x7C
+    B_np[:, 5] = np.where(np.arange(N) % 2 == 0, 0x00, B_np[:, 5])      # Inf * 0 on even columns of row 50
+    got, ref, _ = _run(A_np, E5, api.MAJOR_K, B_np, E4, api.MAJOR_K, M, N, K, torch.float32, want_amax=False)
+    assert np.isnan(ref[20]).all() and np.isnan(ref[:, 40]).all() and np.isinf(ref[3]).any()
+    # K = 0 writes zeros, amax 0; M*N = 0 is a no-op
+    D = torch.full((64, 64), 5.0, dtype=torch.bfloat16, device=DEV)
+    amax = _scalar(9.0)
+    A0 = torch.empty((64, 0), dtype=torch.uint8, device=DEV)
+    B0 = torch.empty((64, 0), dtype=torch.uint8, device=DEV)
+    api.fp8_gemm(A0, E4, api.MAJOR_K, B0, E4, api.MAJOR_K, D, _scalar(1.0), _scalar(1.0), amax)
+    assert bool((D == 0).all()) and amax.item() == 0.0
+    amax.fill_(9.0)
+    Dz = torch.empty((0, 64), dtype=torch.bfloat16, device=DEV)
+    Az = torch.empty((0, 32), dtype=torch.uint8, device=DEV)
+    Bz = torch.empty((64, 32), dtype=torch.uint8, device=DEV)
+    api.fp8_gemm(Az, E4, api.MAJOR_K, Bz, E4, api.MAJOR_K, Dz, _scalar(1.0), _scalar(1.0), amax)
+    assert amax.item() == 0.0
