@@ -36,7 +36,8 @@
  *   - scale multiply and conversion are two roundings (fp32 product, then FP8);
  *   - the special-value rule is applied to the scaled fp32 value, in both
  *     overflow modes (a scaled value of +-Inf is never saturated);
- *   - the NaN emitted is sign | 0x7F in both formats;
+ *   - the NaN emitted is sign | 0x7F in both formats, the sign being that of the
+ *     input element (the sign of a NaN product is not defined by IEEE 754);
  *   - the sign of zero, and of anything that rounds to zero, is kept.
  */
 #include <math.h>
@@ -184,15 +185,24 @@ uint8_t fp8o_encode(float y, int fmt, int overflow)
  * (48 significant bits), so the cast performs the single rounding. */
 static float mul_f32(float a, float b) { return (float)((double)a * (double)b); }
 
+/* One element: scale, then convert.  IEEE 754 leaves the sign of a NaN result of
+ * a multiplication unspecified (processors differ), so the NaN code takes the
+ * sign of the input element x: "the sign of the input is kept". */
+static uint8_t quantize_one(float x, float scale, int fmt, int overflow)
+{
+    float y = mul_f32(x, scale);
+    if (isnan(y)) return (uint8_t)((signbit(x) ? 0x80u : 0u) | 0x7Fu);
+    return fp8o_encode(y, fmt, overflow);
+}
+
 void fp8o_quantize_f32(const float* x, size_t n, float scale, int fmt, int overflow, uint8_t* out)
 {
-    for (size_t i = 0; i < n; ++i) out[i] = fp8o_encode(mul_f32(x[i], scale), fmt, overflow);
+    for (size_t i = 0; i < n; ++i) out[i] = quantize_one(x[i], scale, fmt, overflow);
 }
 
 void fp8o_quantize_bf16(const uint16_t* x, size_t n, float scale, int fmt, int overflow, uint8_t* out)
 {
-    for (size_t i = 0; i < n; ++i)
-        out[i] = fp8o_encode(mul_f32(bf16_to_f32(x[i]), scale), fmt, overflow);
+    for (size_t i = 0; i < n; ++i) out[i] = quantize_one(bf16_to_f32(x[i]), scale, fmt, overflow);
 }
 
 void fp8o_dequantize_f32(const uint8_t* c, size_t n, int fmt, float scale_inv, float* out)

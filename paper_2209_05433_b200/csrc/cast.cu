@@ -111,10 +111,14 @@ __device__ __forceinline__ uint2 quantize_item_bf16(const uint4& v, float scale)
         c.x = cvt_quad<FMT>(y[0], y[1], y[2], y[3]);
         c.y = cvt_quad<FMT>(y[4], y[5], y[6], y[7]);
     } else {
-        c.x = encode_scalar<FMT, NOSAT>(y[0]) | (encode_scalar<FMT, NOSAT>(y[1]) << 8) |
-              (encode_scalar<FMT, NOSAT>(y[2]) << 16) | (encode_scalar<FMT, NOSAT>(y[3]) << 24);
-        c.y = encode_scalar<FMT, NOSAT>(y[4]) | (encode_scalar<FMT, NOSAT>(y[5]) << 8) |
-              (encode_scalar<FMT, NOSAT>(y[6]) << 16) | (encode_scalar<FMT, NOSAT>(y[7]) << 24);
+        uint32_t code[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {                       // sign of x: bit 15 (low half) / bit 31 (high half)
+            code[2 * i] = encode_scaled<FMT, NOSAT>(y[2 * i], w[i] << 16);
+            code[2 * i + 1] = encode_scaled<FMT, NOSAT>(y[2 * i + 1], w[i]);
+        }
+        c.x = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
+        c.y = code[4] | (code[5] << 8) | (code[6] << 16) | (code[7] << 24);
     }
     return c;
 }
@@ -125,8 +129,8 @@ __device__ __forceinline__ uint32_t quantize_item_f32(const uint4& v, float scal
     float y[4] = {__uint_as_float(v.x) * scale, __uint_as_float(v.y) * scale,
                   __uint_as_float(v.z) * scale, __uint_as_float(v.w) * scale};
     if (!needs_scalar_path<FMT, NOSAT>(y)) return cvt_quad<FMT>(y[0], y[1], y[2], y[3]);
-    return encode_scalar<FMT, NOSAT>(y[0]) | (encode_scalar<FMT, NOSAT>(y[1]) << 8) |
-           (encode_scalar<FMT, NOSAT>(y[2]) << 16) | (encode_scalar<FMT, NOSAT>(y[3]) << 24);
+    return encode_scaled<FMT, NOSAT>(y[0], v.x) | (encode_scaled<FMT, NOSAT>(y[1], v.y) << 8) |
+           (encode_scaled<FMT, NOSAT>(y[2], v.z) << 16) | (encode_scaled<FMT, NOSAT>(y[3], v.w) << 24);
 }
 
 // ---------------------------------------------------------------------------
@@ -207,7 +211,8 @@ k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale
             const uint32_t b = scalar_abs_bits<WIDE>(x, i);
             m = WIDE == kWideBF16 ? __vmaxu2(m, b >> 16) : max(m, b);    // bf16 keeps two packed 16-bit lanes
         }
-        out[i] = (uint8_t)encode_scalar<FMT, NOSAT>(scalar_load<WIDE>(x, i) * scale);
+        const float xf = scalar_load<WIDE>(x, i);
+        out[i] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * scale, __float_as_uint(xf));
     }
     if (WITH_AMAX) block_atomic_max_bits(finish_abs_max<WIDE>(m), red, amax_bits);
 }
@@ -296,7 +301,8 @@ k_quantize_elementwise(const void* __restrict__ x, size_t n, const float* __rest
     uint32_t m = 0;
     for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (size_t)gridDim.x * kThreads) {
         if (WITH_AMAX) m = max(m, scalar_abs_bits<WIDE>(x, i));
-        out[i] = (uint8_t)encode_scalar<FMT, NOSAT>(scalar_load<WIDE>(x, i) * scale);
+        const float xf = scalar_load<WIDE>(x, i);
+        out[i] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * scale, __float_as_uint(xf));
     }
     if (WITH_AMAX) block_atomic_max_bits(canonical_nan_bits(m), red, amax_bits);
 }

@@ -62,6 +62,14 @@ __device__ __forceinline__ uint32_t encode_scalar(float y) {
     return sign | mag;
 }
 
+// Scaled value y of input element x -> code.  The multiply does not keep the sign
+// of a NaN operand on this hardware, so a NaN code takes its sign from x.
+template <int FMT, bool NOSAT>
+__device__ __forceinline__ uint32_t encode_scaled(float y, uint32_t x_sign_bit31) {
+    if (y != y) return ((x_sign_bit31 >> 24) & 0x80u) | 0x7Fu;
+    return encode_scalar<FMT, NOSAT>(y);
+}
+
 // Two binary32 values -> two codes (lo in bits 0..7, hi in bits 8..15), hardware RNE,
 // finite overflow saturated.  Only valid for finite inputs (callers check).
 template <int FMT>

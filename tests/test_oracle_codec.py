@@ -290,6 +290,10 @@ def test_quantize_is_fp32_multiply_then_encode(fmt):
     xs = np.array([1e-30, -1e-30, 3e-38], dtype=np.float32)
     ys = xs * np.float32(1e-10)
     assert np.array_equal(oracle.quantize(xs, np.float32(1e-10), fmt), _brute_force_encode(ys, fmt, SATURATE))
+    # a NaN element keeps its own sign, whatever the multiply would make of it
+    nans = np.array([0x7FC00000, 0xFFC00000, 0xFF800001, 0x7FFFFFFF], dtype=np.uint32).view(np.float32)
+    assert oracle.quantize(nans, scale, fmt).tolist() == [0x7F, 0xFF, 0xFF, 0x7F]
+    assert oracle.quantize(nans, np.float32(-2.0), fmt).tolist() == [0x7F, 0xFF, 0xFF, 0x7F]
     # bf16 input widens exactly
     xb = torch.from_numpy(x).to(torch.bfloat16)
     bits = xb.view(torch.int16).numpy().view(np.uint16)
