@@ -1,0 +1,442 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 hot path on B200.
+
+One "step" is one pass of the whole hot path over one synthetic batch of a
+transformer linear layer (hidden 4096 -> 16384, 8192 tokens): for each of the
+activations X, weights W (E4M3) and output gradients dY (E5M2) the two-pass
+current scaling  amax -> scale -> quantize, one dequantize (the FP8 -> bf16
+round trip), then the three FP8 GEMMs with fp32 accumulation and bf16 output
+with epilogue amax: forward Y = X.W, dgrad dX = dY.W^T, wgrad dW = X^T.dY.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is whole-job TFLOP/s: GEMM flops of all ranks
+divided by the max-over-ranks device time of the K steps, casts included.
+`--impl reference` times the CPU oracle (the slow checker under oracle/) on a
+bounded sample of the same step instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fp8_linear_step_gemm_tflops"
+UNIT = "TFLOP/s"
+WORKLOAD = ("transformer linear layer fwd+bwd, hidden 4096->16384, 8192 tokens: amax+scale+quantize of X,W (E4M3) and dY (E5M2), "
+            "one dequantize, fprop/dgrad/wgrad FP8 GEMMs, bf16 out + epilogue amax")
+TOKENS, D_IN, D_OUT, W_SIGMA = 8192, 4096, 16384, 0.02
+NOMINAL_FP8_TFLOPS = 4500.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def peaks():
+    """measured roofline denominators (generated file), else the documented fallback"""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_burst=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    except Exception:
+        return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------
+# clocks sampling
+# ----------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [c for c, p in zip(sm, power) if p >= 0.5 * max(power)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------
+# the step on the GPU
+# ----------------------------------------------------------------------------
+
+class LinearStep:
+    """Buffers and call sequence of one step.  Everything the step computes runs in the library's kernels."""
+
+    def __init__(self, torch, api, synth, device, seed, tokens=TOKENS, d_in=D_IN, d_out=D_OUT):
+        self.torch, self.api = torch, api
+        self.T, self.I, self.O = tokens, d_in, d_out
+        dev = device
+        bf, u8, f32 = torch.bfloat16, torch.uint8, torch.float32
+        self.X = synth.activations(tokens * d_in, seed, dtype=bf, device=dev).view(tokens, d_in)
+        self.W = synth.weights(d_in * d_out, seed, W_SIGMA, dtype=bf, device=dev).view(d_in, d_out)
+        self.dY = synth.gradients(tokens * d_out, seed + 1, dtype=bf, device=dev).view(tokens, d_out)
+        self.Xq = torch.empty(tokens, d_in, dtype=u8, device=dev)
+        self.Wq = torch.empty(d_in, d_out, dtype=u8, device=dev)
+        self.dYq = torch.empty(tokens, d_out, dtype=u8, device=dev)
+        self.Xhat = torch.empty(tokens, d_in, dtype=bf, device=dev)
+        self.Y = torch.empty(tokens, d_out, dtype=bf, device=dev)
+        self.dX = torch.empty(tokens, d_in, dtype=bf, device=dev)
+        self.dW = torch.empty(d_in, d_out, dtype=bf, device=dev)
+        self.scal = torch.zeros(16, dtype=f32, device=dev)      # amax / scale / scale_inv per tensor, GEMM amaxes
+        s = [self.scal[i:i + 1] for i in range(16)]
+        self.ax, self.sx, self.six, self.aw, self.sw, self.siw, self.ag, self.sg, self.sig = s[:9]
+        self.ay, self.adx, self.adw = s[9:12]
+        self.gemm_flops = 3 * 2.0 * tokens * d_in * d_out
+        # algorithmic HBM bytes of the cast part: two-pass (read, read, write) = 5 B per bf16 element; dequantize 3 B
+        n_cast = tokens * d_in + d_in * d_out + tokens * d_out
+        self.cast_bytes = 5.0 * n_cast + 3.0 * tokens * d_in
+
+    def calls(self):
+        """(label, thunk) for every library call of one step, in order"""
+        a = self.api
+        E4, E5, KM, MN = a.E4M3, a.E5M2, a.MAJOR_K, a.MAJOR_MN
+        return [
+            ("amax", lambda: a.fp8_amax(self.X, self.ax)),
+            ("scale", lambda: a.fp8_scale_from_amax(self.ax, E4, self.sx, self.six)),
+            ("quantize", lambda: a.fp8_quantize(self.X, E4, self.sx, self.Xq)),
+            ("amax", lambda: a.fp8_amax(self.W, self.aw)),
+            ("scale", lambda: a.fp8_scale_from_amax(self.aw, E4, self.sw, self.siw)),
+            ("quantize", lambda: a.fp8_quantize(self.W, E4, self.sw, self.Wq)),
+            ("amax", lambda: a.fp8_amax(self.dY, self.ag)),
+            ("scale", lambda: a.fp8_scale_from_amax(self.ag, E5, self.sg, self.sig)),
+            ("quantize", lambda: a.fp8_quantize(self.dY, E5, self.sg, self.dYq)),
+            ("dequantize", lambda: a.fp8_dequantize(self.Xq, E4, self.six, self.Xhat)),
+            # forward: Y[T,O] = X[T,I] . W[I,O]   (W stored with the output index contiguous)
+            ("gemm_fprop", lambda: a.fp8_gemm(self.Xq, E4, KM, self.Wq, E4, MN, self.Y, self.six, self.siw, self.ay)),
+            # dgrad: dX[T,I] = dY[T,O] . W^T      (W stored [I,O] is the [N,K] layout here)
+            ("gemm_dgrad", lambda: a.fp8_gemm(self.dYq, E5, KM, self.Wq, E4, KM, self.dX, self.sig, self.siw, self.adx)),
+            # wgrad: dW[I,O] = X^T . dY           (both operands stored with the contraction index outermost)
+            ("gemm_wgrad", lambda: a.fp8_gemm(self.Xq, E4, MN, self.dYq, E5, MN, self.dW, self.six, self.sig, self.adw)),
+        ]
+
+    def run(self):
+        for _, f in self.calls():
+            f()
+
+    def run_timed(self, events):
+        """one step with a CUDA event before each call and one after the last"""
+        torch = self.torch
+        row = []
+        for label, f in self.calls():
+            e = torch.cuda.Event(enable_timing=True)
+            e.record()
+            row.append((label, e))
+            f()
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        row.append(("end", e))
+        events.append(row)
+
+
+def bench_cast_sweep(torch, api, synth, device, log2n, iters=5):
+    """config-2 style bandwidth point: bf16 tensor of 2^log2n elements; single-pass quantize+amax, amax, dequantize"""
+    n = 1 << log2n
+    x = synth.normal_laplace_mixture(n, 1, synth.T_ID, device=device)
+    codes = torch.empty(n, dtype=torch.uint8, device=device)
+    back = torch.empty(n, dtype=torch.bfloat16, device=device)
+    sc = torch.tensor([3.0, 1.0 / 3.0, 0.0], dtype=torch.float32, device=device)
+    s, si, a = sc[0:1], sc[1:2], sc[2:3]
+    out = {}
+    cases = {
+        "quantize_e4m3_with_amax": (lambda: api.fp8_quantize(x, api.E4M3, s, codes, api.SATURATE, a), 3.0 * n),
+        "quantize_e5m2_with_amax": (lambda: api.fp8_quantize(x, api.E5M2, s, codes, api.SATURATE, a), 3.0 * n),
+        "amax": (lambda: api.fp8_amax(x, a), 2.0 * n),
+        "dequantize_e4m3": (lambda: api.fp8_dequantize(codes, api.E4M3, si, back), 3.0 * n),
+    }
+    for name, (fn, nbytes) in cases.items():
+        for _ in range(3):
+            fn()
+        times = []
+        for _ in range(iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = statistics.median(times)
+        out[name] = {"ms": round(ms, 4), "gbs": round(nbytes / ms / 1e6, 1)}
+    del x, codes, back
+    torch.cuda.empty_cache()
+    return out
+
+
+# ----------------------------------------------------------------------------
+# the oracle arm (CPU)
+# ----------------------------------------------------------------------------
+
+def oracle_step(sample_tokens: int, threads: int):
+    """The same step at `sample_tokens` tokens (weights at full size), run by the CPU oracle as it stands.
+    Returns (seconds, gemm flops of the sample)."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2209_05433_b200 import synth
+
+    T, I, O = sample_tokens, D_IN, D_OUT
+
+    def bits(t):
+        return t.view(torch.int16).numpy().view(np.uint16)
+
+    X = bits(synth.activations(T * I, 3, dtype=torch.bfloat16))
+    W = bits(synth.weights(I * O, 3, W_SIGMA, dtype=torch.bfloat16))
+    dY = bits(synth.gradients(T * O, 4, dtype=torch.bfloat16))
+    t0 = time.perf_counter()
+    q, sinv = {}, {}
+    for name, t, fmt in (("x", X, oracle.E4M3), ("w", W, oracle.E4M3), ("g", dY, oracle.E5M2)):
+        s, si = oracle.scale_from_amax(oracle.amax(t, threads), fmt)
+        q[name], sinv[name] = oracle.quantize(t, s, fmt, threads=threads), si
+    oracle.dequantize(q["x"], sinv["x"], oracle.E4M3, "bf16", threads=threads)
+    y, _ = oracle.gemm_rows(q["x"], oracle.E4M3, (I, 1), q["w"], oracle.E4M3, (O, 1), O, I, 0, T, sinv["x"], sinv["w"], threads)
+    dx, _ = oracle.gemm_rows(q["g"], oracle.E5M2, (O, 1), q["w"], oracle.E4M3, (1, O), I, O, 0, T, sinv["g"], sinv["w"], threads)
+    dw, _ = oracle.gemm_rows(q["x"], oracle.E4M3, (1, I), q["g"], oracle.E5M2, (O, 1), O, T, 0, I, sinv["x"], sinv["g"], threads)
+    for r in (y, dx, dw):
+        oracle.round_bf16_from_f64(r)
+    dt = time.perf_counter() - t0
+    return dt, 3 * 2.0 * T * I * O
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    threads = os.cpu_count() or 1
+    sample_tokens = 8
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(1, threads)
+    times, flops = [], 0.0
+    for _ in range(args.steps):
+        dt, flops = oracle_step(sample_tokens, threads)
+        times.append(dt)
+    total = sum(times)
+    value = flops * len(times) / total / 1e12
+    sample = "the same step with %d of the %d tokens (weights at full size), CPU oracle as it stands" % (sample_tokens, TOKENS)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64 accumulation over decoded fp8 codes", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2209_05433_b200 import api, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    device = "cuda:%d" % local
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    api.load()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # independent batches per rank: no data-path collective (per-tensor amax is local to a rank's own tensors)
+    step = LinearStep(torch, api, synth, device, seed=3 + 16 * rank)
+    for _ in range(max(args.warmup, 3)):
+        step.run()
+    barrier()
+    st, detail = api.fp8_async_status()
+    if st != 0:
+        raise SystemExit("device-side wait expired during warm-up (code %d)" % detail)
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = api.fp8_launch_count()
+    events = []
+    barrier()
+    for _ in range(args.steps):
+        step.run_timed(events)
+    barrier()
+    launches = api.fp8_launch_count() - launches0
+    total_ms = events[0][0][1].elapsed_time(events[-1][-1][1])
+    per_label = {}
+    for row in events:
+        for (label, e0), (_, e1) in zip(row[:-1], row[1:]):
+            per_label.setdefault(label, []).append(e0.elapsed_time(e1))
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    clocks = sampler.stop() if rank == 0 else None
+    st, detail = api.fp8_async_status()
+    if st != 0:
+        raise SystemExit("device-side wait expired during the timed region (code %d)" % detail)
+
+    # ---- end to end: pinned host inputs -> device, the step, results -> pinned host, every step
+    host_in = [torch.empty(t.shape, dtype=t.dtype).pin_memory().copy_(t) for t in (step.X, step.W, step.dY)]
+    host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (step.Y, step.dX, step.dW)]
+    host_scal = torch.empty(16, dtype=torch.float32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = sum(t.numel() * t.element_size() for t in host_out) + host_scal.numel() * 4
+
+    def e2e_step():
+        for h, d in zip(host_in, (step.X, step.W, step.dY)):
+            d.copy_(h, non_blocking=True)
+        step.run()
+        for h, d in zip(host_out, (step.Y, step.dX, step.dW)):
+            h.copy_(d, non_blocking=True)
+        host_scal.copy_(step.scal, non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    if rank == 0:
+        pk = peaks()
+        ms_per_step = total_ms / args.steps
+        value = step.gemm_flops * world / (ms_per_step * 1e-3) / 1e12
+        avg = {k: sum(v) / len(v) for k, v in per_label.items()}
+        calls_per_step = {k: len(v) // args.steps for k, v in per_label.items()}
+        step_sum = sum(avg[k] * calls_per_step[k] for k in avg)
+        kernels = {k: {"avg_ms": round(avg[k], 4), "calls_per_step": calls_per_step[k],
+                       "share": round(avg[k] * calls_per_step[k] / step_sum, 4)} for k in avg}
+        # dominant kernel: the FP8 GEMM (three launches per step of 2*T*I*O flops each)
+        gemm_ms = (avg["gemm_fprop"] + avg["gemm_dgrad"] + avg["gemm_wgrad"]) / 3.0
+        gemm_flops = 2.0 * TOKENS * D_IN * D_OUT
+        achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12
+        fp8_peak = 2.0 * pk["bf16_sustained"]            # fp8 : bf16 nominal ratio is 2
+        roofline = {"bound": "tensor", "kernel": "k_gemm_fp8", "achieved": round(achieved, 1), "peak": round(fp8_peak, 1),
+                    "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4), "traffic": None,
+                    "peak_source": "2 x %s bf16 sustained cuBLAS TFLOP/s (fp8:bf16 nominal ratio)" % pk["source"],
+                    "frac_of_nominal_4500": round(achieved / NOMINAL_FP8_TFLOPS, 4),
+                    "per_gemm_tflops": {k: round(gemm_flops / (avg[k] * 1e-3) / 1e12, 1) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}}
+        # the memory-bound half: amax + quantize (+ dequantize) of the step against HBM
+        cast_ms = sum(avg[k] * calls_per_step[k] for k in ("amax", "scale", "quantize", "dequantize"))
+        cast_gbs = step.cast_bytes / (cast_ms * 1e-3) / 1e9
+        n_x = TOKENS * D_IN + D_IN * D_OUT + TOKENS * D_OUT
+        roofline_cast = {"bound": "hbm", "kernel": "k_amax + k_quantize + k_dequantize (in step)", "achieved": round(cast_gbs, 1),
+                         "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": round(cast_gbs / pk["hbm_gbs"], 4), "traffic": None,
+                         "peak_source": pk["source"] + " copy bandwidth", "frac_of_nominal_8000": round(cast_gbs / NOMINAL_HBM_GBS, 4),
+                         "amax_gbs": round(2.0 * n_x / 3 / (avg["amax"] * 1e-3) / 1e9, 1),
+                         "quantize_gbs": round(3.0 * n_x / 3 / (avg["quantize"] * 1e-3) / 1e9, 1)}
+        cast = None
+        if not args.no_cast_sweep:
+            cast = bench_cast_sweep(torch, api, synth, device, args.cast_log2n)
+            for v in cast.values():
+                v["frac_of_measured_hbm"] = round(v["gbs"] / pk["hbm_gbs"], 4)
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            threads = os.cpu_count() or 1
+            dt, flops = oracle_step(8, threads)
+            cpu = {"value": flops / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": round(dt, 2),
+                   "sample": "the same step with 8 of the %d tokens (weights at full size), CPU oracle as it stands" % TOKENS}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "fp8 (e4m3/e5m2) operands, f32 accumulate, bf16 out", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens": TOKENS, "d_in": D_IN, "d_out": D_OUT, "parallelism": "dp%d" % world,
+                       "l2": "inputs larger than L2 (step touches > 1 GB)", "weights_layout": "[d_in, d_out] row-major"},
+            "clocks": clocks,
+            "e2e": {"value": step.gemm_flops * world / (e2e_ms / e2e_steps * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
+            "gpu_launches": int(launches), "gpu_launches_note": "kernels plus 4-byte memset nodes enqueued by the library in the timed region",
+            "roofline": roofline, "roofline_cast": roofline_cast, "kernels": kernels, "cast_sweep_2pow%d" % args.cast_log2n: cast,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cast-sweep", action="store_true")
+    ap.add_argument("--cast-log2n", type=int, default=28)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
