@@ -160,9 +160,10 @@ class LinearStep:
             ("gemm_wgrad", lambda: a.fp8_gemm(self.Xq, E4, MN, self.dYq, E5, MN, self.dW, self.six, self.sig, self.adw)),
         ]
 
-    def run(self):
-        for _, f in self.calls():
-            f()
+    def run(self, only=None):
+        for label, f in self.calls():
+            if only is None or label == only:
+                f()
 
     def run_timed(self, events):
         """one step with a CUDA event before each call and one after the last"""
@@ -302,6 +303,20 @@ def run_ours(args):
 
     # independent batches per rank: no data-path collective (per-tensor amax is local to a rank's own tensors)
     step = LinearStep(torch, api, synth, device, seed=3 + 16 * rank)
+    if args.only:
+        # profiling aid: one full step to set the scales and codes, then only the named call, timed alone
+        step.run()
+        for _ in range(max(args.warmup, 1)):
+            step.run(args.only)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step.run(args.only)
+        e1.record()
+        torch.cuda.synchronize()
+        print(json.dumps({"only": args.only, "steps": args.steps, "ms_per_step": e0.elapsed_time(e1) / args.steps}))
+        return
     for _ in range(max(args.warmup, 3)):
         step.run()
     barrier()
@@ -425,12 +440,13 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cast-sweep", action="store_true")
     ap.add_argument("--cast-log2n", type=int, default=28)
+    ap.add_argument("--only", default=None, help="profiling aid: time only the calls with this label (e.g. gemm_fprop, quantize, amax)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

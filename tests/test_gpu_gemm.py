@@ -161,7 +161,7 @@ def test_same_sign_accumulation_bound():
         api.fp8_gemm(A, E4, api.MAJOR_K, B, E4, api.MAJOR_K, D, _scalar(1.0), _scalar(1.0))
         torch.cuda.synchronize()
         assert api.fp8_async_status()[0] == 0
-        ref, sabs = oracle.gemm_rows(A_np, E4, (K, 1), B_np, E4, (K, 1), N, K, 0, M, 1.0, 1.0, threads=THREADS)
+        ref, sabs = oracle.gemm_rows(A_np, E4, (K, 1), B_np, E4, (1, K), N, K, 0, M, 1.0, 1.0, threads=THREADS)
         rel = np.abs(to_np_bits(D).astype(np.float64) - ref) / sabs
         bound = 1e-5 if K <= 2048 else (K / 32) * 2.0 ** -23
         assert rel.max() <= bound, (K, rel.max(), bound)
