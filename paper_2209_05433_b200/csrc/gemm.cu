@@ -2,26 +2,34 @@
 // the paper: dot products of FP8 inputs accumulated in binary32, unscaled once
 // per dot product, written in a wider type.
 //
-// One persistent CTA per SM works through 128 x 256 output tiles.
-//   warp 0       TMA producer: cp.async.bulk.tensor loads of A (128 x 128 B) and
-//                B (256 x 128 B) K-blocks into a 4-stage 128B-swizzled smem ring
-//   warp 1       TMEM allocation, and one elected lane issuing tcgen05.mma
-//                (kind::f8f6f4, M128 N256 K32) into one of two 256-column TMEM
-//                accumulators; tcgen05.commit releases smem stages / publishes
-//                the finished accumulator
+// One persistent CTA per SM.  CG (CTA group) = 2: the two CTAs of a cluster
+// work on one 256 x 256 output tile, each holding 128 rows of A, half of the B
+// tile and its own 128 x 256 accumulator; the leader CTA issues
+// tcgen05.mma.cta_group::2 (M256 N256 K32) for both.  That halves the B bytes
+// each SM stages and reads per flop.  CG = 1 (128 x 256 tiles, one CTA) serves
+// problems with at most 128 rows.
+//   warp 0       TMA producer: cp.async.bulk.tensor loads of this CTA's A rows
+//                and B rows into a 128B-swizzled smem ring; completion is
+//                signalled on the leader CTA's "full" barrier
+//   warp 1       TMEM allocation (both CTAs) and, in the leader, one lane issuing
+//                the MMAs into one of two 256-column TMEM accumulators;
+//                tcgen05.commit releases the smem stage in both CTAs / publishes
+//                the finished accumulator to both CTAs' epilogues
 //   warps 2..5   epilogue: tcgen05.ld of the accumulator (each warp owns its 32
 //                TMEM lanes), multiply by sa_inv*sb_inv, round to bf16 / keep
 //                fp32, amax of the stored values, global stores.  The epilogue
 //                of tile i overlaps the main loop of tile i+1.
 // Operands may be K-major or MN-major (forward / dgrad / wgrad layouts); the
 // two formats of a mixed E5M2 x E4M3 product are set in the instruction
-// descriptor.  No TMA multicast is used anywhere.
-// Every mbarrier wait is bounded: on expiry the kernel latches an error code,
+// descriptor.  No TMA load uses cluster multicast.
+// Every mbarrier wait is bounded (about 2 s): on expiry the kernel latches an error code,
 // all roles drain, TMEM is freed and the kernel returns.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "codec.cuh"
@@ -33,24 +41,43 @@ __device__ unsigned int g_async_latch[2] = {0u, 0u};
 
 namespace gemm {
 
+#ifdef FP8_GEMM_PROFILE
+// Development aid, absent from the product build: per-CTA cycle counters of where each role waits.
+__device__ unsigned long long g_prof[512 * 8];
+#define PROF_DECL long long prof_t = 0, prof_acc0 = 0, prof_acc1 = 0; const long long prof_start = clock64();
+#define PROF_BEGIN prof_t = clock64();
+#define PROF_END(acc) acc += clock64() - prof_t;
+#define PROF_STORE(slot0, slot1, slot2) if (lane == 0) { g_prof[blockIdx.x * 8 + slot0] = prof_acc0; g_prof[blockIdx.x * 8 + slot1] = prof_acc1; if (slot2 >= 0) g_prof[blockIdx.x * 8 + slot2] = clock64() - prof_start; }
+#else
+#define PROF_DECL
+#define PROF_BEGIN
+#define PROF_END(acc)
+#define PROF_STORE(slot0, slot1, slot2)
+#endif
+
 constexpr int BM = 128;             // tile rows  (= UMMA M, one TMEM lane per row)
 constexpr int BN = 256;             // tile cols  (= UMMA N, one TMEM column per col)
 constexpr int BK = 128;             // K-block in elements = bytes = one 128B swizzle row
 constexpr int UMMA_K = 32;          // K of one tcgen05.mma for 8-bit operands
-constexpr int STAGES = 4;
+constexpr int MAX_STAGES = 6;
 constexpr int ACC_STAGES = 2;       // 2 x 256 columns = all 512 TMEM columns
 constexpr int THREADS = 192;
 constexpr int EPI_WARPS = 4;
-constexpr uint32_t A_BYTES = BM * BK;          // 16 KiB
-constexpr uint32_t B_BYTES = BN * BK;          // 32 KiB
-constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr uint32_t SMEM_TILES = STAGES * STAGE_BYTES;
+constexpr uint32_t A_BYTES = BM * BK;          // 16 KiB: this CTA's 128 rows of A
+// per CTA group size: B bytes staged by one CTA, stage size, ring depth (192 KiB of tiles either way)
+template <int CG> struct Geo {
+    static constexpr uint32_t B_BYTES = (BN / CG) * BK;             // 32 KiB alone, 16 KiB when paired
+    static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = CG == 1 ? 4 : 6;
+    static constexpr int TILE_M = BM * CG;
+};
+constexpr uint32_t SMEM_TILES = 4 * (A_BYTES + BN * BK);            // = 6 * (A_BYTES + BN/2 * BK)
 constexpr uint32_t SMEM_BARRIERS = 256;
 constexpr uint32_t SMEM_BYTES = SMEM_TILES + SMEM_BARRIERS + 1024;   // + slack to align the ring to 1024 B
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int GROUP_M = 8;          // tile raster: GROUP_M row-tiles share each sweep over N
 
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clocks per wait
 
 // codes written to the error latch
 enum : uint32_t { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC_EMPTY = 3, WAIT_ACC_FULL = 4 };
@@ -77,29 +104,64 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait.  Returns false after WAIT_LIMIT_NS, or at once when another
-// role has already given up (abort flag), having latched `code`.
+// Bounded wait.  Returns false after about WAIT_LIMIT_CYCLES SM clocks (checked every 1024 failed
+// polls, so that the common short wait never reads a timer), or as soon as another role of this CTA
+// has given up (abort flag), having latched `code`.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    uint32_t spins = 0;
-    while (true) {
+    long long t0 = 0;
+    for (uint32_t spins = 1;; ++spins) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 255u) == 0u) {
+        if ((spins & 1023u) == 0u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_CYCLES) {
                 *abort_flag = 1u;
                 if (atomicCAS(&g_async_latch[0], 0u, code) == 0u) g_async_latch[1] = blockIdx.x;
                 return false;
             }
         }
     }
+}
+
+// cluster (CTA pair) helpers
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {     // same variable in CTA `rank`
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+// TMA load whose completion is counted on a barrier that may live in the peer CTA of the pair
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t cluster_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar) : "memory");
+}
+// commit of a CTA-pair MMA: arrives on the barrier at this offset in both CTAs
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_f8_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -155,13 +217,13 @@ struct Params {
     const float* sa_inv;
     const float* sb_inv;
     uint32_t* amax_bits;            // may be null
-    uint32_t idesc;
-    int tiles_m, tiles_n;
+    uint32_t idesc;                 // M field set for the CTA group the kernel was built for
+    int tiles_m, tiles_n;           // tiles of (128*CG) x 256
 };
 
 struct alignas(8) Barriers {
-    uint64_t full[STAGES];
-    uint64_t empty[STAGES];
+    uint64_t full[MAX_STAGES];
+    uint64_t empty[MAX_STAGES];
     uint64_t acc_full[ACC_STAGES];
     uint64_t acc_empty[ACC_STAGES];
     uint32_t tmem_base;
@@ -181,11 +243,14 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
     tn = r / rows;
 }
 
-// A_MN / B_MN: operand stored with its M (resp. N) index contiguous.
+// CG: CTAs per tile (1 or 2).  A_MN / B_MN: operand stored with its M (resp. N) index contiguous.
 // OUT_BF16: D is bf16, else fp32.
-template <bool A_MN, bool B_MN, bool OUT_BF16>
+template <int CG, bool A_MN, bool B_MN, bool OUT_BF16>
 __global__ void __launch_bounds__(THREADS, 1)
 k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params p) {
+    using G = Geo<CG>;
+    constexpr int STAGES = G::STAGES;
+    constexpr uint32_t STAGE_BYTES = G::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;                 // 1024-byte aligned tile ring
@@ -194,67 +259,94 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    const uint32_t cta_rank = CG == 2 ? cluster_ctarank() : 0u;   // 0 = leader of the pair
+    const int worker = blockIdx.x / CG, num_workers = gridDim.x / CG;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int k_blocks = (int)((p.K + BK - 1) / BK);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), 1); mbar_init(smem_u32(&bars->empty[s]), 1); }
-        for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(smem_u32(&bars->acc_full[a]), 1); mbar_init(smem_u32(&bars->acc_empty[a]), EPI_WARPS); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), CG); mbar_init(smem_u32(&bars->empty[s]), 1); }
+        for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(smem_u32(&bars->acc_full[a]), 1); mbar_init(smem_u32(&bars->acc_empty[a]), EPI_WARPS * CG); }
         bars->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {                                              // whole warp: allocate all 512 TMEM columns
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (warp == 1) {                                              // whole warp (of each CTA): all 512 TMEM columns
+        if (CG == 2) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();                              // the peer's barriers are initialised too
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ TMA producer (each CTA loads its own rows)
         uint32_t stage = 0, phase = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        PROF_DECL
+        for (int t = worker; t < num_tiles && ok; t += num_workers) {
             int tm, tn;
             tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
-            const int m0 = tm * BM, n0 = tn * BN;
+            const int m0 = tm * G::TILE_M + (int)cta_rank * BM;                 // this CTA's 128 rows of A
+            const int n0 = tn * BN + (int)cta_rank * (BN / CG);                 // this CTA's rows of B
             for (int kb = 0; kb < k_blocks; ++kb) {
+                PROF_BEGIN
                 ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, WAIT_EMPTY);
+                PROF_END(prof_acc0)
                 if (!ok) break;
                 if (lane == 0) {
-                    const uint32_t full = smem_u32(&bars->full[stage]);
                     const uint32_t sa = ring + stage * STAGE_BYTES;
                     const uint32_t sb = sa + A_BYTES;
                     const int k0 = kb * BK;
-                    mbar_arrive_expect_tx(full, STAGE_BYTES);
-                    if (A_MN) tma_load_2d(sa, &map_a, m0, k0, full);          // box {128 m, 128 k}
-                    else      tma_load_2d(sa, &map_a, k0, m0, full);          // box {128 k, 128 m}
-                    if (B_MN) {                                               // two boxes {128 n, 128 k}
-                        tma_load_2d(sb, &map_b, n0, k0, full);
-                        tma_load_2d(sb + B_BYTES / 2, &map_b, n0 + 128, k0, full);
+                    if (CG == 2) {
+                        const uint32_t full = map_to_cta(smem_u32(&bars->full[stage]), 0);   // the leader's barrier
+                        mbar_arrive_expect_tx_cluster(full, STAGE_BYTES);
+                        if (A_MN) tma_load_2d_pair(sa, &map_a, m0, k0, full);     // box {128 m, 128 k}
+                        else      tma_load_2d_pair(sa, &map_a, k0, m0, full);     // box {128 k, 128 m}
+                        if (B_MN) tma_load_2d_pair(sb, &map_b, n0, k0, full);     // box {128 n, 128 k}
+                        else      tma_load_2d_pair(sb, &map_b, k0, n0, full);     // box {128 k, 128 n}
                     } else {
-                        tma_load_2d(sb, &map_b, k0, n0, full);                // box {128 k, 256 n}
+                        const uint32_t full = smem_u32(&bars->full[stage]);
+                        mbar_arrive_expect_tx(full, STAGE_BYTES);
+                        if (A_MN) tma_load_2d(sa, &map_a, m0, k0, full);
+                        else      tma_load_2d(sa, &map_a, k0, m0, full);
+                        if (B_MN) {                                               // two boxes {128 n, 128 k}
+                            tma_load_2d(sb, &map_b, n0, k0, full);
+                            tma_load_2d(sb + G::B_BYTES / 2, &map_b, n0 + 128, k0, full);
+                        } else {
+                            tma_load_2d(sb, &map_b, k0, n0, full);                // box {128 k, 256 n}
+                        }
                     }
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
+        PROF_STORE(0, 1, 2)
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
         uint32_t stage = 0, phase = 0;
-        bool ok = true;
+        bool ok = cta_rank == 0;
         int it = 0;
-        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+        PROF_DECL
+        for (int t = worker; t < num_tiles && ok; t += num_workers, ++it) {
             const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
+            PROF_BEGIN
             ok = mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag, WAIT_ACC_EMPTY);
+            PROF_END(prof_acc1)
             if (!ok) break;
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * BN;
             for (int kb = 0; kb < k_blocks; ++kb) {
+                PROF_BEGIN
                 ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, WAIT_FULL);
+                PROF_END(prof_acc0)
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
@@ -268,30 +360,41 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                                                  : smem_desc(sa + k * UMMA_K, 16, 1024);
                         const uint64_t db = B_MN ? smem_desc(sb + k * UMMA_K * 128, BK * 128, 1024)
                                                  : smem_desc(sb + k * UMMA_K, 16, 1024);
-                        tc_mma_f8(tmem_d, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                        if (CG == 2) tc_mma_f8_pair(tmem_d, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                        else         tc_mma_f8(tmem_d, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    tc_commit(smem_u32(&bars->empty[stage]));                 // frees the smem stage when the MMAs retire
-                    if (kb == k_blocks - 1) tc_commit(smem_u32(&bars->acc_full[acc]));
+                    // frees the smem stage (in both CTAs) when the MMAs retire; the last block also publishes the accumulator
+                    if (CG == 2) {
+                        tc_commit_pair(smem_u32(&bars->empty[stage]));
+                        if (kb == k_blocks - 1) tc_commit_pair(smem_u32(&bars->acc_full[acc]));
+                    } else {
+                        tc_commit(smem_u32(&bars->empty[stage]));
+                        if (kb == k_blocks - 1) tc_commit(smem_u32(&bars->acc_full[acc]));
+                    }
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
+        PROF_STORE(3, 4, 5)
     } else {
-        // ------------------------------------------------------------ epilogue
+        // ------------------------------------------------------------ epilogue (each CTA drains its own 128 rows)
         const int q = warp & 3;                                   // TMEM lane quarter this warp may read
         const float alpha = __ldg(p.sa_inv) * __ldg(p.sb_inv);
         uint32_t running = 0;                                     // max of stored magnitude bits (bf16: 16-bit patterns)
         bool ok = true;
         int it = 0;
-        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+        PROF_DECL
+        for (int t = worker; t < num_tiles && ok; t += num_workers, ++it) {
             int tm, tn;
             tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
             const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
+            PROF_BEGIN
             ok = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, WAIT_ACC_FULL);
+            PROF_END(prof_acc0)
             if (!ok) break;
             tc_fence_after();
-            const int64_t row = (int64_t)tm * BM + q * 32 + lane;
+            const int64_t row = (int64_t)tm * G::TILE_M + cta_rank * BM + q * 32 + lane;
             const int64_t col0 = (int64_t)tn * BN;
             const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
@@ -348,8 +451,12 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[acc]));      // accumulator may be overwritten
+            if (lane == 0) {                                      // accumulator may be overwritten: tell the leader's MMA warp
+                if (CG == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0));
+                else         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
+            }
         }
+        if (warp == 2) { PROF_STORE(6, 7, -1) }
         if (p.amax_bits) {
             uint32_t bits = OUT_BF16 ? (max(running & 0xFFFFu, running >> 16) << 16) : running;
             bits = warp_max_u32(canonical_nan_bits(bits));
@@ -359,9 +466,11 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
 
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();        // neither CTA leaves while the other may still touch its smem, barriers or TMEM
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        if (CG == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        else         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -409,14 +518,44 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool A_MN, bool B_MN, bool OUT_BF16>
-static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid, cudaStream_t st) {
-    auto k = k_gemm_fp8<A_MN, B_MN, OUT_BF16>;
+// CTA-pair kernels launch as clusters of 2; the grid is one CTA per SM that can be paired.
+template <int CG, bool A_MN, bool B_MN, bool OUT_BF16>
+static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int64_t num_tiles, cudaStream_t st) {
+    auto k = k_gemm_fp8<CG, A_MN, B_MN, OUT_BF16>;
     // per device and cheap, so set on every launch rather than cached
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return FP8_ERR_CUDA;
-    k<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(THREADS, 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int workers = sm_count() / CG;
+    if (CG == 2) {
+        cfg.gridDim = dim3(2 * workers, 1, 1);
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, k, &cfg) == cudaSuccess && clusters > 0 && clusters < workers) workers = clusters;
+    }
+    if ((int64_t)workers > num_tiles) workers = (int)num_tiles;
+    cfg.gridDim = dim3(workers * CG, 1, 1);
+    if (getenv("FP8_B200_DEBUG")) fprintf(stderr, "[fp8_b200] gemm CG=%d grid=%d tiles=%lld\n", CG, workers * CG, (long long)num_tiles);
+    if (cudaLaunchKernelEx(&cfg, k, ma, mb, p) != cudaSuccess) return FP8_ERR_CUDA;
     count_launches(1);
     return launch_status();
+}
+
+template <int CG>
+static fp8_status dispatch(bool a_mn, bool b_mn, bool bf, const CUtensorMap& ma, const CUtensorMap& mb, const Params& p,
+                           int64_t num_tiles, cudaStream_t st) {
+    if (!a_mn && !b_mn) return bf ? launch<CG, false, false, true>(ma, mb, p, num_tiles, st) : launch<CG, false, false, false>(ma, mb, p, num_tiles, st);
+    if (!a_mn && b_mn)  return bf ? launch<CG, false, true, true>(ma, mb, p, num_tiles, st)  : launch<CG, false, true, false>(ma, mb, p, num_tiles, st);
+    if (a_mn && !b_mn)  return bf ? launch<CG, true, false, true>(ma, mb, p, num_tiles, st)  : launch<CG, true, false, false>(ma, mb, p, num_tiles, st);
+    return bf ? launch<CG, true, true, true>(ma, mb, p, num_tiles, st) : launch<CG, true, true, false>(ma, mb, p, num_tiles, st);
 }
 
 }  // namespace gemm
@@ -439,7 +578,10 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
     cudaStream_t st = (cudaStream_t)stream;
     const bool a_mn = d->ma == FP8_MAJOR_MN, b_mn = d->mb == FP8_MAJOR_MN;
     const int64_t esz = d->out == FP8_BF16 ? 2 : 4;
-    const int64_t tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
+    // CTA pairs (256-row tiles) unless the whole problem has at most 128 rows
+    const int cg = M > BM ? 2 : 1;
+    const int64_t tile_m = (int64_t)BM * cg;
+    const int64_t tiles_m = (M + tile_m - 1) / tile_m, tiles_n = (N + BN - 1) / BN;
     // ---- validation: nothing is enqueued before every check has passed
     if (M > 0 && N > 0) {
         if (!D) return FP8_ERR_NULL;
@@ -470,10 +612,11 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
     }
 
     CUtensorMap map_a, map_b;
+    const uint32_t b_rows = (uint32_t)(BN / cg);                  // B rows one CTA loads per K-block
     bool ok = a_mn ? make_map(&map_a, A, (uint64_t)M, (uint64_t)K, (uint64_t)d->lda, 128, BK)
                    : make_map(&map_a, A, (uint64_t)K, (uint64_t)M, (uint64_t)d->lda, BK, BM);
     ok = ok && (b_mn ? make_map(&map_b, B, (uint64_t)N, (uint64_t)K, (uint64_t)d->ldb, 128, BK)
-                     : make_map(&map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)d->ldb, BK, BN));
+                     : make_map(&map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)d->ldb, BK, b_rows));
     if (!ok) return FP8_ERR_CUDA;
 
     Params p;
@@ -481,17 +624,20 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
     p.sa_inv = scale_inv_a_dev; p.sb_inv = scale_inv_b_dev;
     p.amax_bits = reinterpret_cast<uint32_t*>(amax_d_dev);
     p.tiles_m = (int)tiles_m; p.tiles_n = (int)tiles_n;
-    // instruction descriptor: fp32 accumulate, operand formats and majors, N/8, M/16
+    // instruction descriptor: fp32 accumulate, operand formats and majors, N/8, M/16 (M = 256 for a CTA pair)
     p.idesc = (1u << 4) | ((uint32_t)d->fa << 7) | ((uint32_t)d->fb << 10) | ((a_mn ? 1u : 0u) << 15) |
-              ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-    int grid = sm_count();
-    if ((int64_t)grid > tiles_m * tiles_n) grid = (int)(tiles_m * tiles_n);
+              ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
     const bool bf = d->out == FP8_BF16;
-    if (!a_mn && !b_mn) return bf ? launch<false, false, true>(map_a, map_b, p, grid, st) : launch<false, false, false>(map_a, map_b, p, grid, st);
-    if (!a_mn && b_mn)  return bf ? launch<false, true, true>(map_a, map_b, p, grid, st)  : launch<false, true, false>(map_a, map_b, p, grid, st);
-    if (a_mn && !b_mn)  return bf ? launch<true, false, true>(map_a, map_b, p, grid, st)  : launch<true, false, false>(map_a, map_b, p, grid, st);
-    return bf ? launch<true, true, true>(map_a, map_b, p, grid, st) : launch<true, true, false>(map_a, map_b, p, grid, st);
+    return cg == 2 ? dispatch<2>(a_mn, b_mn, bf, map_a, map_b, p, tiles_m * tiles_n, st)
+                   : dispatch<1>(a_mn, b_mn, bf, map_a, map_b, p, tiles_m * tiles_n, st);
 }
+
+#ifdef FP8_GEMM_PROFILE
+int fp8_debug_gemm_profile(unsigned long long* host_out, int n) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(host_out, fp8b200::gemm::g_prof, sizeof(unsigned long long) * n);
+}
+#endif
 
 fp8_status fp8_async_status(uint32_t* detail) {
     unsigned int latch[2] = {0u, 0u};
