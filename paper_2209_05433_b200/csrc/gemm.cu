@@ -17,8 +17,9 @@
 //                the finished accumulator to both CTAs' epilogues
 //   warps 2..5   epilogue: tcgen05.ld of the accumulator (each warp owns its 32
 //                TMEM lanes), multiply by sa_inv*sb_inv, round to bf16 / keep
-//                fp32, amax of the stored values, global stores.  The epilogue
-//                of tile i overlaps the main loop of tile i+1.
+//                fp32, amax of the stored values, swizzled staging in shared
+//                memory and TMA tensor stores (edges clipped by the TMA unit).
+//                The epilogue of tile i overlaps the main loop of tile i+1.
 // Operands may be K-major or MN-major (forward / dgrad / wgrad layouts); the
 // two formats of a mixed E5M2 x E4M3 product are set in the instruction
 // descriptor.  No TMA load uses cluster multicast.
@@ -72,8 +73,10 @@ template <int CG> struct Geo {
     static constexpr int TILE_M = BM * CG;
 };
 constexpr uint32_t SMEM_TILES = 4 * (A_BYTES + BN * BK);            // = 6 * (A_BYTES + BN/2 * BK)
+constexpr uint32_t EPI_BUF_BYTES = 4096;                            // 32 rows x 128 B, one TMA store box
+constexpr uint32_t SMEM_EPI = EPI_WARPS * 2 * EPI_BUF_BYTES;        // two staging buffers per epilogue warp
 constexpr uint32_t SMEM_BARRIERS = 256;
-constexpr uint32_t SMEM_BYTES = SMEM_TILES + SMEM_BARRIERS + 1024;   // + slack to align the ring to 1024 B
+constexpr uint32_t SMEM_BYTES = SMEM_TILES + SMEM_EPI + SMEM_BARRIERS + 1024;   // + slack to align the ring to 1024 B
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int GROUP_M = 8;          // tile raster: GROUP_M row-tiles share each sweep over N
 
@@ -146,10 +149,10 @@ __device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_a
     asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
 }
 // TMA load whose completion is counted on a barrier that may live in the peer CTA of the pair
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t cluster_bar) {
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t cluster_bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar) : "memory");
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar), "l"(policy) : "memory");
 }
 // commit of a CTA-pair MMA: arrives on the barrier at this offset in both CTAs
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
@@ -164,10 +167,34 @@ __device__ __forceinline__ void tc_mma_f8_pair(uint32_t tmem_d, uint64_t adesc, 
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy) : "memory");
+}
+// L2 eviction policies: operand panels are re-read by many CTAs (keep), the output is written once (stream)
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+// TMA tensor store of one staged box, tracked by the issuing thread's bulk async-group
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -247,14 +274,15 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 // OUT_BF16: D is bf16, else fp32.
 template <int CG, bool A_MN, bool B_MN, bool OUT_BF16>
 __global__ void __launch_bounds__(THREADS, 1)
-k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params p) {
+k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+           const __grid_constant__ CUtensorMap map_d, const Params p) {
     using G = Geo<CG>;
     constexpr int STAGES = G::STAGES;
     constexpr uint32_t STAGE_BYTES = G::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;                 // 1024-byte aligned tile ring
-    Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (ring - raw) + SMEM_TILES);
+    Barriers* bars = reinterpret_cast<Barriers*>(smem_raw + (ring - raw) + SMEM_TILES + SMEM_EPI);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5;
@@ -289,6 +317,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         // ------------------------------------------------------------ TMA producer (each CTA loads its own rows)
         uint32_t stage = 0, phase = 0;
         bool ok = true;
+        const uint64_t keep = policy_evict_last();
         PROF_DECL
         for (int t = worker; t < num_tiles && ok; t += num_workers) {
             int tm, tn;
@@ -307,20 +336,20 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     if (CG == 2) {
                         const uint32_t full = map_to_cta(smem_u32(&bars->full[stage]), 0);   // the leader's barrier
                         mbar_arrive_expect_tx_cluster(full, STAGE_BYTES);
-                        if (A_MN) tma_load_2d_pair(sa, &map_a, m0, k0, full);     // box {128 m, 128 k}
-                        else      tma_load_2d_pair(sa, &map_a, k0, m0, full);     // box {128 k, 128 m}
-                        if (B_MN) tma_load_2d_pair(sb, &map_b, n0, k0, full);     // box {128 n, 128 k}
-                        else      tma_load_2d_pair(sb, &map_b, k0, n0, full);     // box {128 k, 128 n}
+                        if (A_MN) tma_load_2d_pair(sa, &map_a, m0, k0, full, keep);     // box {128 m, 128 k}
+                        else      tma_load_2d_pair(sa, &map_a, k0, m0, full, keep);     // box {128 k, 128 m}
+                        if (B_MN) tma_load_2d_pair(sb, &map_b, n0, k0, full, keep);     // box {128 n, 128 k}
+                        else      tma_load_2d_pair(sb, &map_b, k0, n0, full, keep);     // box {128 k, 128 n}
                     } else {
                         const uint32_t full = smem_u32(&bars->full[stage]);
                         mbar_arrive_expect_tx(full, STAGE_BYTES);
-                        if (A_MN) tma_load_2d(sa, &map_a, m0, k0, full);
-                        else      tma_load_2d(sa, &map_a, k0, m0, full);
+                        if (A_MN) tma_load_2d(sa, &map_a, m0, k0, full, keep);
+                        else      tma_load_2d(sa, &map_a, k0, m0, full, keep);
                         if (B_MN) {                                               // two boxes {128 n, 128 k}
-                            tma_load_2d(sb, &map_b, n0, k0, full);
-                            tma_load_2d(sb + G::B_BYTES / 2, &map_b, n0 + 128, k0, full);
+                            tma_load_2d(sb, &map_b, n0, k0, full, keep);
+                            tma_load_2d(sb + G::B_BYTES / 2, &map_b, n0 + 128, k0, full, keep);
                         } else {
-                            tma_load_2d(sb, &map_b, k0, n0, full);                // box {128 k, 256 n}
+                            tma_load_2d(sb, &map_b, k0, n0, full, keep);                // box {128 k, 256 n}
                         }
                     }
                 }
@@ -382,6 +411,9 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         const int q = warp & 3;                                   // TMEM lane quarter this warp may read
         const float alpha = __ldg(p.sa_inv) * __ldg(p.sb_inv);
         uint32_t running = 0;                                     // max of stored magnitude bits (bf16: 16-bit patterns)
+        const uint32_t epi_base = ring + SMEM_TILES + (uint32_t)(warp - 2) * 2u * EPI_BUF_BYTES;
+        uint32_t buf = 0;
+        const uint64_t stream_out = policy_evict_first();
         bool ok = true;
         int it = 0;
         PROF_DECL
@@ -394,60 +426,72 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             PROF_END(prof_acc0)
             if (!ok) break;
             tc_fence_after();
-            const int64_t row = (int64_t)tm * G::TILE_M + cta_rank * BM + q * 32 + lane;
+            const int row0 = tm * G::TILE_M + (int)cta_rank * BM + q * 32;      // first of this warp's 32 rows
+            const bool row_ok = (int64_t)row0 + lane < p.M;
             const int64_t col0 = (int64_t)tn * BN;
             const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+            constexpr int CHUNK = OUT_BF16 ? 64 : 32;             // columns per staged box: 128 bytes per row
+            constexpr int ESZ = OUT_BF16 ? 2 : 4;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                tc_ld32(taddr + c * 32, r);
-                tc_wait_ld();
-                const int64_t col = col0 + c * 32;
-                if (row < p.M && col < p.N) {
-                    const bool full_chunk = col + 32 <= p.N;
-                    if (OUT_BF16) {
-                        uint16_t* dst = reinterpret_cast<uint16_t*>(p.D) + row * p.ldd + col;
-                        uint32_t w[16];
+            for (int c = 0; c < BN / CHUNK; ++c) {
+                uint32_t w[32];                                   // the 128 bytes this thread contributes to its row
+                if (OUT_BF16) {
+                    uint32_t r0[32], r1[32];
+                    tc_ld32(taddr + c * 64, r0);
+                    tc_ld32(taddr + c * 64 + 32, r1);
+                    tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            w[i] = pack_bf16(__uint_as_float(r[2 * i]) * alpha, __uint_as_float(r[2 * i + 1]) * alpha);
-                        }
-                        if (full_chunk) {
+                    for (int i = 0; i < 16; ++i) {
+                        w[i] = pack_bf16(__uint_as_float(r0[2 * i]) * alpha, __uint_as_float(r0[2 * i + 1]) * alpha);
+                        w[16 + i] = pack_bf16(__uint_as_float(r1[2 * i]) * alpha, __uint_as_float(r1[2 * i + 1]) * alpha);
+                    }
+                } else {
+                    tc_ld32(taddr + c * 32, w);
+                    tc_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) running = __vmaxu2(running, w[i] & 0x7FFF7FFFu);
+                    for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
+                }
+                const int64_t col = col0 + (int64_t)c * CHUNK;
+                if (row_ok && col < p.N) {                        // amax over in-bounds elements only
+                    if (col + CHUNK <= p.N) {
 #pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-                        } else {
-                            for (int i = 0; i < 32 && col + i < p.N; ++i) {
-                                const uint32_t h = (i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu);
-                                running = __vmaxu2(running, h & 0x7FFFu);
-                                dst[i] = (uint16_t)h;
-                            }
-                        }
+                        for (int i = 0; i < 32; ++i)
+                            running = OUT_BF16 ? __vmaxu2(running, w[i] & 0x7FFF7FFFu) : max(running, w[i] & 0x7FFFFFFFu);
                     } else {
-                        float* dst = reinterpret_cast<float*>(p.D) + row * p.ldd + col;
-                        if (full_chunk) {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                float4 v;
-                                v.x = __uint_as_float(r[4 * i]) * alpha;
-                                v.y = __uint_as_float(r[4 * i + 1]) * alpha;
-                                v.z = __uint_as_float(r[4 * i + 2]) * alpha;
-                                v.w = __uint_as_float(r[4 * i + 3]) * alpha;
-                                running = max(running, max(max(__float_as_uint(v.x) & 0x7FFFFFFFu, __float_as_uint(v.y) & 0x7FFFFFFFu),
-                                                           max(__float_as_uint(v.z) & 0x7FFFFFFFu, __float_as_uint(v.w) & 0x7FFFFFFFu)));
-                                reinterpret_cast<float4*>(dst)[i] = v;
-                            }
-                        } else {
-                            for (int i = 0; i < 32 && col + i < p.N; ++i) {
-                                const float v = __uint_as_float(r[i]) * alpha;
-                                running = max(running, __float_as_uint(v) & 0x7FFFFFFFu);
-                                dst[i] = v;
-                            }
+                        for (int i = 0; i < CHUNK && col + i < p.N; ++i) {
+                            const uint32_t h = OUT_BF16 ? (((i & 1) ? (w[i >> 1] >> 16) : w[i >> 1]) & 0x7FFFu) : (w[i] & 0x7FFFFFFFu);
+                            running = OUT_BF16 ? __vmaxu2(running, h) : max(running, h);
                         }
                     }
                 }
+                // A box that crosses the right edge is clipped by the TMA unit in 16-byte units: when the row
+                // length in bytes is not a multiple of 16 that last box is written with plain stores instead.
+                const bool clipped_mid_16 = col + CHUNK > p.N && ((p.N * ESZ) & 15) != 0;
+                if (clipped_mid_16) {
+                    if (row_ok) {
+                        for (int i = 0; i < CHUNK && col + i < p.N; ++i) {
+                            if (OUT_BF16) reinterpret_cast<uint16_t*>(p.D)[((int64_t)row0 + lane) * p.ldd + col + i] =
+                                              (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : w[i >> 1]);
+                            else          reinterpret_cast<uint32_t*>(p.D)[((int64_t)row0 + lane) * p.ldd + col + i] = w[i];
+                        }
+                    }
+                    continue;
+                }
+                // stage the 32 x 128 B box with the 128-byte swizzle the tensor map expects, then store it
+                if (lane == 0) bulk_wait_read<1>();               // the box stored two chunks ago has left this buffer
+                __syncwarp();
+                const uint32_t sbuf = epi_base + buf * EPI_BUF_BYTES;
+                const uint32_t srow = sbuf + lane * 128;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    st_shared_v4(srow + ((j ^ (lane & 7)) << 4), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (row0 < p.M && col < p.N) tma_store_2d(&map_d, sbuf, (int)(col * ESZ), row0, stream_out);
+                    bulk_commit();
+                }
+                buf ^= 1u;
             }
             tc_fence_before();
             __syncwarp();
@@ -456,6 +500,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 else         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
             }
         }
+        if (lane == 0) bulk_wait_all();                           // every store has reached global memory before exit
         if (warp == 2) { PROF_STORE(6, 7, -1) }
         if (p.amax_bits) {
             uint32_t bits = OUT_BF16 ? (max(running & 0xFFFFu, running >> 16) << 16) : running;
@@ -520,7 +565,7 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
 
 // CTA-pair kernels launch as clusters of 2; the grid is one CTA per SM that can be paired.
 template <int CG, bool A_MN, bool B_MN, bool OUT_BF16>
-static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int64_t num_tiles, cudaStream_t st) {
+static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const Params& p, int64_t num_tiles, cudaStream_t st) {
     auto k = k_gemm_fp8<CG, A_MN, B_MN, OUT_BF16>;
     // per device and cheap, so set on every launch rather than cached
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return FP8_ERR_CUDA;
@@ -544,18 +589,18 @@ static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const Par
     if ((int64_t)workers > num_tiles) workers = (int)num_tiles;
     cfg.gridDim = dim3(workers * CG, 1, 1);
     if (getenv("FP8_B200_DEBUG")) fprintf(stderr, "[fp8_b200] gemm CG=%d grid=%d tiles=%lld\n", CG, workers * CG, (long long)num_tiles);
-    if (cudaLaunchKernelEx(&cfg, k, ma, mb, p) != cudaSuccess) return FP8_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, k, ma, mb, md, p) != cudaSuccess) return FP8_ERR_CUDA;
     count_launches(1);
     return launch_status();
 }
 
 template <int CG>
-static fp8_status dispatch(bool a_mn, bool b_mn, bool bf, const CUtensorMap& ma, const CUtensorMap& mb, const Params& p,
-                           int64_t num_tiles, cudaStream_t st) {
-    if (!a_mn && !b_mn) return bf ? launch<CG, false, false, true>(ma, mb, p, num_tiles, st) : launch<CG, false, false, false>(ma, mb, p, num_tiles, st);
-    if (!a_mn && b_mn)  return bf ? launch<CG, false, true, true>(ma, mb, p, num_tiles, st)  : launch<CG, false, true, false>(ma, mb, p, num_tiles, st);
-    if (a_mn && !b_mn)  return bf ? launch<CG, true, false, true>(ma, mb, p, num_tiles, st)  : launch<CG, true, false, false>(ma, mb, p, num_tiles, st);
-    return bf ? launch<CG, true, true, true>(ma, mb, p, num_tiles, st) : launch<CG, true, true, false>(ma, mb, p, num_tiles, st);
+static fp8_status dispatch(bool a_mn, bool b_mn, bool bf, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
+                           const Params& p, int64_t num_tiles, cudaStream_t st) {
+    if (!a_mn && !b_mn) return bf ? launch<CG, false, false, true>(ma, mb, md, p, num_tiles, st) : launch<CG, false, false, false>(ma, mb, md, p, num_tiles, st);
+    if (!a_mn && b_mn)  return bf ? launch<CG, false, true, true>(ma, mb, md, p, num_tiles, st)  : launch<CG, false, true, false>(ma, mb, md, p, num_tiles, st);
+    if (a_mn && !b_mn)  return bf ? launch<CG, true, false, true>(ma, mb, md, p, num_tiles, st)  : launch<CG, true, false, false>(ma, mb, md, p, num_tiles, st);
+    return bf ? launch<CG, true, true, true>(ma, mb, md, p, num_tiles, st) : launch<CG, true, true, false>(ma, mb, md, p, num_tiles, st);
 }
 
 }  // namespace gemm
@@ -617,6 +662,9 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
                    : make_map(&map_a, A, (uint64_t)K, (uint64_t)M, (uint64_t)d->lda, BK, BM);
     ok = ok && (b_mn ? make_map(&map_b, B, (uint64_t)N, (uint64_t)K, (uint64_t)d->ldb, 128, BK)
                      : make_map(&map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)d->ldb, BK, b_rows));
+    // D as a byte tensor {N*esz, M}: boxes of 128 bytes x 32 rows, the unit each epilogue warp stores
+    CUtensorMap map_d;
+    ok = ok && make_map(&map_d, D, (uint64_t)(N * esz), (uint64_t)M, (uint64_t)(d->ldd * esz), 128, 32);
     if (!ok) return FP8_ERR_CUDA;
 
     Params p;
@@ -628,8 +676,8 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
     p.idesc = (1u << 4) | ((uint32_t)d->fa << 7) | ((uint32_t)d->fb << 10) | ((a_mn ? 1u : 0u) << 15) |
               ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
     const bool bf = d->out == FP8_BF16;
-    return cg == 2 ? dispatch<2>(a_mn, b_mn, bf, map_a, map_b, p, tiles_m * tiles_n, st)
-                   : dispatch<1>(a_mn, b_mn, bf, map_a, map_b, p, tiles_m * tiles_n, st);
+    return cg == 2 ? dispatch<2>(a_mn, b_mn, bf, map_a, map_b, map_d, p, tiles_m * tiles_n, st)
+                   : dispatch<1>(a_mn, b_mn, bf, map_a, map_b, map_d, p, tiles_m * tiles_n, st);
 }
 
 #ifdef FP8_GEMM_PROFILE
