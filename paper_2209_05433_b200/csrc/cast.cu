@@ -35,7 +35,49 @@ int sm_count() {
 
 constexpr int kWideF32 = 0;
 constexpr int kWideBF16 = 1;
-constexpr int kThreads = 256;
+#ifndef FP8_CAST_THREADS
+#define FP8_CAST_THREADS 256
+#endif
+#ifndef FP8_QUANT_UNROLL_BF16
+#define FP8_QUANT_UNROLL_BF16 2
+#endif
+#ifndef FP8_DEQUANT_UNROLL
+#define FP8_DEQUANT_UNROLL 4
+#endif
+#ifndef FP8_AMAX_UNROLL
+#define FP8_AMAX_UNROLL 8
+#endif
+constexpr int kThreads = FP8_CAST_THREADS;
+
+// Output stores: written once, never re-read by the same kernel.
+__device__ __forceinline__ void st_out(uint2* p, uint2 v) {
+#ifdef FP8_STORE_CS
+    __stcs(p, v);
+#else
+    *p = v;
+#endif
+}
+__device__ __forceinline__ void st_out(uint32_t* p, uint32_t v) {
+#ifdef FP8_STORE_CS
+    __stcs(p, v);
+#else
+    *p = v;
+#endif
+}
+__device__ __forceinline__ void st_out(uint4* p, uint4 v) {
+#ifdef FP8_STORE_CS
+    __stcs(p, v);
+#else
+    *p = v;
+#endif
+}
+__device__ __forceinline__ void st_out(float4* p, float4 v) {
+#ifdef FP8_STORE_CS
+    __stcs(p, v);
+#else
+    *p = v;
+#endif
+}
 
 // ---------------------------------------------------------------------------
 // per-item arithmetic
@@ -185,8 +227,8 @@ k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale
 
     auto emit = [&](size_t i, const uint4& v) {
         if (WITH_AMAX) m = fold_abs_max<WIDE>(m, v);
-        if (WIDE == kWideBF16) reinterpret_cast<uint2*>(out)[i] = quantize_item_bf16<FMT, NOSAT>(v, scale);
-        else                   reinterpret_cast<uint32_t*>(out)[i] = quantize_item_f32<FMT, NOSAT>(v, scale);
+        if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out) + i, quantize_item_bf16<FMT, NOSAT>(v, scale));
+        else                   st_out(reinterpret_cast<uint32_t*>(out) + i, quantize_item_f32<FMT, NOSAT>(v, scale));
     };
 
     for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
@@ -235,11 +277,11 @@ k_dequantize(const uint8_t* __restrict__ c, size_t n, const float* __restrict__ 
         o.y = pack_bf16(b.x * si, b.y * si);
         o.z = pack_bf16(d.x * si, d.y * si);
         o.w = pack_bf16(e.x * si, e.y * si);
-        reinterpret_cast<uint4*>(out)[i] = o;
+        st_out(reinterpret_cast<uint4*>(out) + i, o);
     };
     auto emit_f32 = [&](size_t i, uint32_t w) {
         const float2 a = decode_pair<FMT>(w), b = decode_pair<FMT>(w >> 16);
-        reinterpret_cast<float4*>(out)[i] = make_float4(a.x * si, a.y * si, b.x * si, b.y * si);
+        st_out(reinterpret_cast<float4*>(out) + i, make_float4(a.x * si, a.y * si, b.x * si, b.y * si));
     };
 
     for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
@@ -353,10 +395,10 @@ static size_t chunks_of(size_t n, int epi, int unroll) {
     return (items + per_chunk - 1) / per_chunk;
 }
 
-constexpr int kAmaxUnroll = 8;
-constexpr int kQuantUnrollBF16 = 4;
+constexpr int kAmaxUnroll = FP8_AMAX_UNROLL;
+constexpr int kQuantUnrollBF16 = FP8_QUANT_UNROLL_BF16;
 constexpr int kQuantUnrollF32 = 8;
-constexpr int kDequantUnroll = 4;
+constexpr int kDequantUnroll = FP8_DEQUANT_UNROLL;
 
 template <int WIDE>
 static fp8_status launch_amax(const void* x, size_t n, uint32_t* bits, cudaStream_t st) {

@@ -78,7 +78,7 @@ constexpr uint32_t SMEM_EPI = EPI_WARPS * 2 * EPI_BUF_BYTES;        // two stagi
 constexpr uint32_t SMEM_BARRIERS = 256;
 constexpr uint32_t SMEM_BYTES = SMEM_TILES + SMEM_EPI + SMEM_BARRIERS + 1024;   // + slack to align the ring to 1024 B
 constexpr uint32_t TMEM_COLS = 512;
-constexpr int GROUP_M = 8;          // tile raster: GROUP_M row-tiles share each sweep over N
+constexpr int GROUP_M = 16;         // tile raster: GROUP_M row-tiles share each sweep over N
 
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clocks per wait
 
