@@ -91,6 +91,28 @@ fp8_status fp8_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_o
                         const float* scale_dev, uint8_t* out, float* amax_dev, void* stream);
 
 /*
+ * fp8_quantize_current — Section 2, the whole "current scaling" conversion of one tensor in ONE launch:
+ * the scale is chosen from the tensor's own maximum magnitude, then the tensor is converted with it.
+ * Results are identical, bit for bit, to fp8_amax + fp8_scale_from_amax + fp8_quantize:
+ *   *amax_dev = amax(x); *scale_dev = fmax/amax (same guards); *scale_inv_dev = 1/scale;
+ *   out_i = encode_f( binary32(x_i) * scale ).
+ * The kernel is launched cooperatively (all of its blocks resident at once) and crosses one grid-wide
+ * barrier between the two passes; the second pass re-reads the tail of x from L2.
+ *   workspace  device, fp8_quantize_current_workspace_bytes() bytes, 16-byte aligned, owned by the
+ *              caller.  It must hold zeros before the first call; every call leaves it zeroed again,
+ *              so one buffer serves any number of calls on one stream.  Calls that may overlap on the
+ *              GPU (different streams) need different workspaces.
+ * The grid barrier is a bounded wait: if it expires nothing is written and fp8_async_status reports
+ * FP8_ERR_TIMEOUT (the workspace must then be zeroed again by the caller).
+ */
+fp8_status fp8_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o,
+                                uint8_t* out, float* amax_dev, float* scale_dev, float* scale_inv_dev,
+                                void* workspace, void* stream);
+
+/* Size in bytes of the workspace fp8_quantize_current needs. */
+size_t fp8_quantize_current_workspace_bytes(void);
+
+/*
  * fp8_dequantize — Section 2: convert back and multiply by the inverse of the
  * scale factor.  out_i = round_t( decode_f(c_i) * scale_inv ), one binary32
  * multiply, then round-to-nearest-even to bf16 when t is FP8_BF16.  NaN codes

@@ -19,7 +19,8 @@ F32, BF16 = 0, 1             # fp8_wide
 SATURATE, NOSAT = 0, 1       # fp8_overflow
 MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
 
-EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_dequantize", "fp8_gemm",
+EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
+           "fp8_quantize_current_workspace_bytes", "fp8_dequantize", "fp8_gemm",
            "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
 
 
@@ -62,6 +63,10 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_scale_from_amax.argtypes = [vp, i32, vp, vp, vp]
     lib.fp8_quantize.restype = i32
     lib.fp8_quantize.argtypes = [vp, i32, sz, i32, i32, vp, vp, vp, vp]
+    lib.fp8_quantize_current.restype = i32
+    lib.fp8_quantize_current.argtypes = [vp, i32, sz, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.fp8_quantize_current_workspace_bytes.restype = sz
+    lib.fp8_quantize_current_workspace_bytes.argtypes = []
     lib.fp8_dequantize.restype = i32
     lib.fp8_dequantize.argtypes = [vp, sz, i32, vp, vp, i32, vp]
     lib.fp8_gemm.restype = i32
@@ -123,6 +128,31 @@ def fp8_quantize(x: torch.Tensor, fmt: int, scale: torch.Tensor, out: torch.Tens
     _check(load().fp8_quantize(_dev(x, "x"), _wide_of(x), x.numel(), fmt, overflow, _scalar(scale, "scale"),
                                _dev(out, "out"), None if amax_out is None else _scalar(amax_out, "amax_out"),
                                _stream()), "fp8_quantize")
+
+
+_workspaces: dict = {}
+
+
+def current_scaling_workspace(device: torch.device) -> torch.Tensor:
+    """A zeroed workspace for fp8_quantize_current on `device`, made once per (device, stream)."""
+    key = (device.index if device.index is not None else torch.cuda.current_device(), _stream())
+    ws = _workspaces.get(key)
+    if ws is None:
+        nbytes = int(load().fp8_quantize_current_workspace_bytes())
+        ws = torch.zeros(max(nbytes, 16), dtype=torch.uint8, device=device)
+        _workspaces[key] = ws
+    return ws
+
+
+def fp8_quantize_current(x: torch.Tensor, fmt: int, out: torch.Tensor, amax_out: torch.Tensor, scale_out: torch.Tensor,
+                         scale_inv_out: torch.Tensor, overflow: int = SATURATE, workspace: torch.Tensor | None = None) -> None:
+    if out.dtype != torch.uint8 or out.numel() != x.numel():
+        raise TypeError("out must be a uint8 tensor with as many elements as x")
+    ws = current_scaling_workspace(x.device) if workspace is None else workspace
+    _check(load().fp8_quantize_current(_dev(x, "x"), _wide_of(x), x.numel(), fmt, overflow, _dev(out, "out"),
+                                       _scalar(amax_out, "amax_out"), _scalar(scale_out, "scale_out"),
+                                       _scalar(scale_inv_out, "scale_inv_out"), _dev(ws, "workspace"), _stream()),
+           "fp8_quantize_current")
 
 
 def fp8_dequantize(codes: torch.Tensor, fmt: int, scale_inv: torch.Tensor, out: torch.Tensor) -> None:

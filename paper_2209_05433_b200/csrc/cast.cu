@@ -19,6 +19,9 @@ namespace fp8b200 {
 static std::atomic<uint64_t> g_launches{0};
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o, uint8_t* out,
+                                   float* amax, float* scale, float* scale_inv, unsigned int* ws, cudaStream_t st);
+
 int sm_count() {
     static std::mutex mu;
     static int cached[64] = {0};
@@ -372,6 +375,146 @@ __global__ void k_scale_from_amax(const float* amax_dev, float fmax, float* scal
     *scale_inv_dev = __fdiv_rn(1.0f, s);
 }
 
+// scale and inverse scale from an amax value: the arithmetic of k_scale_from_amax, callable from other kernels
+__device__ __forceinline__ void scale_pair_from_amax(float a, float fmax, float& s, float& si) {
+    s = 1.0f;
+    if (a == a && a != 0.0f && fabsf(a) != __int_as_float(0x7F800000)) {
+        s = __fdiv_rn(fmax, a);
+        if (fabsf(s) == __int_as_float(0x7F800000)) s = __int_as_float(0x7F7FFFFF);
+    }
+    si = __fdiv_rn(1.0f, s);
+}
+
+// Error latch of the cast kernels' bounded waits: [0] = code, [1] = block.
+__device__ unsigned int g_cast_latch[2] = {0u, 0u};
+constexpr unsigned int kWaitGridBarrier = 16u;
+constexpr long long kGridWaitLimitCycles = 4000000000ll;       // about 2 s of SM clocks
+
+// Current scaling in ONE launch: amax of x, scale = fmax / amax, quantize with that scale.
+// All CTAs are co-resident (cooperative launch).  ws[0] = running amax bits, ws[1] = arrivals at the
+// grid barrier, ws[2] = departures; the three words are zero on entry and the last CTA to leave puts
+// them back to zero.  The second pass walks each CTA's chunks in reverse so that the part of x read
+// last in the first pass is re-read from L2.
+template <int WIDE, int FMT, bool NOSAT, int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __restrict__ out,
+                   float* amax_out, float* scale_out, float* scale_inv_out, unsigned int* ws) {
+    __shared__ uint32_t red[32];
+    __shared__ uint32_t bcast[2];
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    const size_t n_items = n / EPI;
+    const size_t per_chunk = (size_t)kThreads * UNROLL;
+    const size_t n_chunks = (n_items + per_chunk - 1) / per_chunk;
+    const size_t tail = n - n_items * EPI;
+
+    // ---- pass 1: amax
+    uint32_t m = 0;
+    for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        const size_t base = chunk * per_chunk + threadIdx.x;
+        if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
+            uint4 v[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) v[u] = *(xv + base + (size_t)u * kThreads);   // default caching: kept in L2 for pass 2
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) m = fold_abs_max<WIDE>(m, v[u]);
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const size_t i = base + (size_t)u * kThreads;
+                if (i < n_items) m = fold_abs_max<WIDE>(m, *(xv + i));
+            }
+        }
+    }
+    m = finish_abs_max<WIDE>(m);
+    if (blockIdx.x == 0 && threadIdx.x < tail)
+        m = max(m, canonical_nan_bits(scalar_abs_bits<WIDE>(x, n_items * EPI + threadIdx.x)));
+    block_atomic_max_bits(m, red, ws);
+
+    // ---- grid barrier (bounded), then every CTA reads the same amax
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&ws[1], 1u);
+        uint32_t okflag = 1u;
+        long long t0 = 0;
+        for (uint32_t spins = 1;; ++spins) {
+            unsigned int arrived;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(arrived) : "l"(&ws[1]) : "memory");
+            if (arrived >= gridDim.x) break;
+            if ((spins & 255u) == 0u) {
+                const long long now = clock64();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kGridWaitLimitCycles) {
+                    if (atomicCAS(&g_cast_latch[0], 0u, kWaitGridBarrier) == 0u) g_cast_latch[1] = blockIdx.x;
+                    okflag = 0u;
+                    break;
+                }
+            }
+        }
+        unsigned int bits;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(bits) : "l"(&ws[0]) : "memory");
+        bcast[0] = bits;
+        bcast[1] = okflag;
+    }
+    __syncthreads();
+    const float amax = __uint_as_float(bcast[0]);
+    const bool ok = bcast[1] != 0u;
+    float scale, scale_inv;
+    scale_pair_from_amax(amax, fmax, scale, scale_inv);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && ok) {
+        *amax_out = amax;
+        *scale_out = scale;
+        *scale_inv_out = scale_inv;
+    }
+
+    // ---- pass 2: quantize, this CTA's chunks in reverse order
+    if (ok && n_chunks > blockIdx.x) {
+        const size_t my_chunks = (n_chunks - blockIdx.x + gridDim.x - 1) / gridDim.x;
+        for (size_t c = my_chunks; c-- > 0;) {
+            const size_t chunk = blockIdx.x + c * gridDim.x;
+            const size_t base = chunk * per_chunk + threadIdx.x;
+            if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
+                uint4 v[UNROLL];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const size_t i = base + (size_t)u * kThreads;
+                    if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out) + i, quantize_item_bf16<FMT, NOSAT>(v[u], scale));
+                    else                   st_out(reinterpret_cast<uint32_t*>(out) + i, quantize_item_f32<FMT, NOSAT>(v[u], scale));
+                }
+            } else {
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const size_t i = base + (size_t)u * kThreads;
+                    if (i < n_items) {
+                        const uint4 v = ld_nc_v4(xv + i);
+                        if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out) + i, quantize_item_bf16<FMT, NOSAT>(v, scale));
+                        else                   st_out(reinterpret_cast<uint32_t*>(out) + i, quantize_item_f32<FMT, NOSAT>(v, scale));
+                    }
+                }
+            }
+        }
+    }
+    if (ok && blockIdx.x == 0 && threadIdx.x < tail) {
+        const size_t i = n_items * EPI + threadIdx.x;
+        const float xf = scalar_load<WIDE>(x, i);
+        out[i] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * scale, __float_as_uint(xf));
+    }
+
+    // ---- leave the workspace as it was found: the last CTA out zeroes it
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int gone = atomicAdd(&ws[2], 1u);
+        if (gone == gridDim.x - 1) {
+            ws[0] = 0u;
+            ws[2] = 0u;
+            __threadfence();
+            ws[1] = 0u;
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
@@ -463,6 +606,46 @@ static fp8_status zero_word(void* p, cudaStream_t st) {
     return FP8_OK;
 }
 
+template <int WIDE, int FMT, bool NOSAT>
+static fp8_status launch_current(const void* x, size_t n, float fmax, uint8_t* out, float* amax, float* scale, float* scale_inv,
+                                 unsigned int* ws, cudaStream_t st) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int UNROLL = 4;
+    auto k = k_quantize_current<WIDE, FMT, NOSAT, UNROLL>;
+    size_t chunks = chunks_of(n, EPI, UNROLL);
+    if (chunks < 1) chunks = 1;
+    const int grid = persistent_grid(k, chunks);               // co-resident by construction: SMs x occupancy at most
+    void* args[] = {(void*)&x, (void*)&n, (void*)&fmax, (void*)&out, (void*)&amax, (void*)&scale, (void*)&scale_inv, (void*)&ws};
+    if (cudaLaunchCooperativeKernel((const void*)k, dim3(grid), dim3(kThreads), args, 0, st) != cudaSuccess) return FP8_ERR_CUDA;
+    count_launches(1);
+    return launch_status();
+}
+
+// The vector path needs x 16-byte aligned and out aligned to the codes one item produces; other
+// alignments take the three separate calls (identical results).
+fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o, uint8_t* out,
+                                   float* amax, float* scale, float* scale_inv, unsigned int* ws, cudaStream_t st) {
+    const int epi = t == FP8_BF16 ? 8 : 4;
+    if (n == 0 || !aligned16(x) || (reinterpret_cast<uintptr_t>(out) & (epi - 1)) != 0) {
+        fp8_status s = fp8_amax(x, t, n, amax, st);
+        if (s == FP8_OK) s = fp8_scale_from_amax(amax, f, scale, scale_inv, st);
+        if (s == FP8_OK) s = fp8_quantize(x, t, n, f, o, scale, out, nullptr, st);
+        return s;
+    }
+    const float fmax = f == FP8_E4M3 ? 448.0f : 57344.0f;
+    const bool nosat = o == FP8_NOSAT;
+    if (t == FP8_F32) {
+        if (f == FP8_E4M3) return nosat ? launch_current<kWideF32, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                        : launch_current<kWideF32, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+        return nosat ? launch_current<kWideF32, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                     : launch_current<kWideF32, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+    }
+    if (f == FP8_E4M3) return nosat ? launch_current<kWideBF16, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                    : launch_current<kWideBF16, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+    return nosat ? launch_current<kWideBF16, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                 : launch_current<kWideBF16, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+}
+
 }  // namespace fp8b200
 
 using namespace fp8b200;
@@ -505,6 +688,27 @@ fp8_status fp8_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_o
                              : dispatch_quantize<kWideF32, kE5M2>(x, n, nosat, scale_dev, out, bits, st);
     return f == FP8_E4M3 ? dispatch_quantize<kWideBF16, kE4M3>(x, n, nosat, scale_dev, out, bits, st)
                          : dispatch_quantize<kWideBF16, kE5M2>(x, n, nosat, scale_dev, out, bits, st);
+}
+
+fp8_status fp8_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o, uint8_t* out,
+                                float* amax_dev, float* scale_dev, float* scale_inv_dev, void* workspace, void* stream) {
+    if (!amax_dev || !scale_dev || !scale_inv_dev || !workspace || ((!x || !out) && n)) return FP8_ERR_NULL;
+    if ((t != FP8_F32 && t != FP8_BF16) || (f != FP8_E4M3 && f != FP8_E5M2) || (o != FP8_SATURATE && o != FP8_NOSAT))
+        return FP8_ERR_ENUM;
+    if (reinterpret_cast<uintptr_t>(workspace) & 15u) return FP8_ERR_ALIGN;
+    return fp8b200::launch_quantize_current(x, t, n, f, o, out, amax_dev, scale_dev, scale_inv_dev,
+                                            reinterpret_cast<unsigned int*>(workspace), (cudaStream_t)stream);
+}
+
+size_t fp8_quantize_current_workspace_bytes(void) { return 16; }
+
+void fp8_cast_read_clear_latch(unsigned int out2[2]) {
+    out2[0] = out2[1] = 0u;
+    if (cudaMemcpyFromSymbol(out2, fp8b200::g_cast_latch, 2 * sizeof(unsigned int)) != cudaSuccess) return;
+    if (out2[0] != 0u) {
+        const unsigned int zero[2] = {0u, 0u};
+        cudaMemcpyToSymbol(fp8b200::g_cast_latch, zero, sizeof(zero));
+    }
 }
 
 fp8_status fp8_dequantize(const uint8_t* c, size_t n, fp8_format f, const float* scale_inv_dev, void* out, fp8_wide t, void* stream) {

@@ -687,10 +687,18 @@ int fp8_debug_gemm_profile(unsigned long long* host_out, int n) {
 }
 #endif
 
+void fp8_cast_read_clear_latch(unsigned int out2[2]);      // defined with the cast kernels
+
 fp8_status fp8_async_status(uint32_t* detail) {
     unsigned int latch[2] = {0u, 0u};
     if (cudaDeviceSynchronize() != cudaSuccess) return FP8_ERR_CUDA;
+    unsigned int cast_latch[2];
+    fp8_cast_read_clear_latch(cast_latch);
     if (cudaMemcpyFromSymbol(latch, g_async_latch, sizeof(latch)) != cudaSuccess) return FP8_ERR_CUDA;
+    if (latch[0] == 0u && cast_latch[0] != 0u) {
+        if (detail) *detail = cast_latch[0];
+        return FP8_ERR_TIMEOUT;
+    }
     if (detail) *detail = latch[0];
     if (latch[0] == 0u) return FP8_OK;
     const unsigned int zero[2] = {0u, 0u};

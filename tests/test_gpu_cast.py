@@ -256,3 +256,44 @@ def test_config2_large_sizes_sampled(log2n):
         del codes, back
     del x
     torch.cuda.empty_cache()
+
+
+# ------------------------------------------ fused current scaling (one launch) --
+
+@pytest.mark.parametrize("wide", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 9, 1000, 4099, (1 << 20) + 3, (1 << 24) + 17])
+def test_quantize_current_equals_three_calls_and_oracle(wide, n):
+    x = synth.activations(n, 3, dtype=wide, device=DEV)
+    x_np = to_np_bits(x)
+    for fmt in FMTS:
+        for overflow in (api.SATURATE, api.NOSAT):
+            a, s, si = _scalar(-1.0), _scalar(-1.0), _scalar(-1.0)
+            out = torch.full((n + 64,), 0xA5, dtype=torch.uint8, device=DEV)
+            for _ in range(2):                                  # twice in a row: the workspace is left clean
+                api.fp8_quantize_current(x, fmt, out[:n], a, s, si, overflow)
+            torch.cuda.synchronize()
+            assert api.fp8_async_status()[0] == 0
+            want_amax_bits = oracle.amax_bits(x_np, THREADS)
+            ws, wsi = oracle.scale_from_amax(np.array([want_amax_bits], dtype=np.uint32).view(np.float32)[0], fmt)
+            assert a.cpu().numpy().view(np.uint32)[0] == want_amax_bits
+            assert s.item() == ws and si.item() == wsi
+            _assert_codes(out[:n].cpu().numpy(), oracle.quantize(x_np, ws, fmt, overflow, threads=THREADS), x_np)
+            assert bool((out[n:] == 0xA5).all())
+            assert bool((api.current_scaling_workspace(x.device) == 0).all())
+
+
+def test_quantize_current_specials_and_unaligned():
+    n = 100003
+    base = synth.normal_laplace_mixture(n + 16, 9, synth.T_ID, dtype=torch.bfloat16, device=DEV)
+    for off, poke in ((0, float("nan")), (0, float("inf")), (3, None)):        # offset 3 takes the three-call path
+        x = base[off: off + n].clone() if off == 0 else base[off: off + n]
+        if poke is not None:
+            x[n // 2] = poke
+        x_np = to_np_bits(x)
+        a, s, si = _scalar(-1.0), _scalar(-1.0), _scalar(-1.0)
+        out = torch.empty(n, dtype=torch.uint8, device=DEV)
+        api.fp8_quantize_current(x, api.E4M3, out, a, s, si)
+        want_bits = oracle.amax_bits(x_np)
+        ws, wsi = oracle.scale_from_amax(np.array([want_bits], dtype=np.uint32).view(np.float32)[0], oracle.E4M3)
+        assert a.cpu().numpy().view(np.uint32)[0] == want_bits and s.item() == ws and si.item() == wsi
+        _assert_codes(out.cpu().numpy(), oracle.quantize(x_np, ws, oracle.E4M3), x_np)
