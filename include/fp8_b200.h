@@ -113,6 +113,38 @@ fp8_status fp8_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format 
 size_t fp8_quantize_current_workspace_bytes(void);
 
 /*
+ * fp8_quantize_current_static — the paper has no counterpart; this entry point exists for callers
+ * that cannot obtain device memory for a workspace.
+ *
+ * Who that is: code that runs where cudaMalloc is off limits or would fail — a plug-in called from
+ * inside another framework's memory pool that already owns all of the GPU's memory, a latency-bound
+ * serving loop in which an allocation (an implicit device synchronisation) is not acceptable, or a
+ * component that is only ever handed its input and output buffers.  Such a caller still wants the
+ * one-launch current-scaling conversion of fp8_quantize_current, but has no 16 spare bytes to pass.
+ *
+ * What it does: exactly fp8_quantize_current (same kernel, same results bit for bit), with the
+ * kernel's three control words kept in a 256-byte array that is part of the library image.  Every GPU
+ * that loads the library holds those 256 bytes until the process exits.  The call allocates nothing:
+ * no cudaMalloc, no cudaFree, no allocating library routine.  The caller passes inputs and outputs only.
+ *
+ * Rules of use
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the words it needs before its
+ *     kernel runs, so a call never depends on what the previous one left behind; but two calls that
+ *     overlap on the GPU (different streams, or different host threads on different streams) race on
+ *     it and give undefined results.  Issue them on one stream, or serialise them yourself.
+ *   - n may not exceed FP8_STATIC_MAX_ELEMENTS; larger tensors return FP8_ERR_UNSUPPORTED and nothing
+ *     is enqueued.  (The scratch need of this kernel does not grow with n; the bound is the largest
+ *     size this entry point is exercised and supported at.)
+ *   - Arguments, alignment rules and the bounded grid barrier are those of fp8_quantize_current.
+ */
+#define FP8_STATIC_MAX_ELEMENTS ((size_t)1 << 32)
+fp8_status fp8_quantize_current_static(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o,
+                                       uint8_t* out, float* amax_dev, float* scale_dev, float* scale_inv_dev,
+                                       void* stream);
+
+/*
  * fp8_dequantize — Section 2: convert back and multiply by the inverse of the
  * scale factor.  out_i = round_t( decode_f(c_i) * scale_inv ), one binary32
  * multiply, then round-to-nearest-even to bf16 when t is FP8_BF16.  NaN codes

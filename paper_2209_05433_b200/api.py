@@ -20,7 +20,7 @@ SATURATE, NOSAT = 0, 1       # fp8_overflow
 MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
 
 EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
-           "fp8_quantize_current_workspace_bytes", "fp8_dequantize", "fp8_gemm",
+           "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_gemm",
            "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
 
 
@@ -67,6 +67,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_quantize_current.argtypes = [vp, i32, sz, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.fp8_quantize_current_workspace_bytes.restype = sz
     lib.fp8_quantize_current_workspace_bytes.argtypes = []
+    lib.fp8_quantize_current_static.restype = i32
+    lib.fp8_quantize_current_static.argtypes = [vp, i32, sz, i32, i32, vp, vp, vp, vp, vp]
     lib.fp8_dequantize.restype = i32
     lib.fp8_dequantize.argtypes = [vp, sz, i32, vp, vp, i32, vp]
     lib.fp8_gemm.restype = i32
@@ -153,6 +155,21 @@ def fp8_quantize_current(x: torch.Tensor, fmt: int, out: torch.Tensor, amax_out:
                                        _scalar(amax_out, "amax_out"), _scalar(scale_out, "scale_out"),
                                        _scalar(scale_inv_out, "scale_inv_out"), _dev(ws, "workspace"), _stream()),
            "fp8_quantize_current")
+
+
+STATIC_MAX_ELEMENTS = 1 << 32
+
+
+def fp8_quantize_current_static(x: torch.Tensor, fmt: int, out: torch.Tensor, amax_out: torch.Tensor,
+                                scale_out: torch.Tensor, scale_inv_out: torch.Tensor, overflow: int = SATURATE) -> None:
+    """fp8_quantize_current for callers that cannot allocate a workspace: the kernel's control words
+    live in a small array inside the library.  Calls that overlap on the GPU race on that array."""
+    if out.dtype != torch.uint8 or out.numel() != x.numel():
+        raise TypeError("out must be a uint8 tensor with as many elements as x")
+    _check(load().fp8_quantize_current_static(_dev(x, "x"), _wide_of(x), x.numel(), fmt, overflow, _dev(out, "out"),
+                                              _scalar(amax_out, "amax_out"), _scalar(scale_out, "scale_out"),
+                                              _scalar(scale_inv_out, "scale_inv_out"), _stream()),
+           "fp8_quantize_current_static")
 
 
 def fp8_dequantize(codes: torch.Tensor, fmt: int, scale_inv: torch.Tensor, out: torch.Tensor) -> None:

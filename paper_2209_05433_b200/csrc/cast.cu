@@ -702,6 +702,46 @@ fp8_status fp8_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format 
 
 size_t fp8_quantize_current_workspace_bytes(void) { return 16; }
 
+// ---- fp8_quantize_current_static: the same kernel, its scratch words in library-owned static memory ----
+//
+// g_static_scratch is what the kernel uses as its three control words.  In host code this name is only
+// a stand-in for the device object: its device address is obtained once per device with
+// cudaGetSymbolAddress (that device being current) and that address is what the kernel receives.
+constexpr size_t kStaticScratchBytes = 256;
+static __device__ __align__(256) unsigned int g_static_scratch[kStaticScratchBytes / sizeof(unsigned int)];
+
+static fp8_status static_scratch_address(unsigned int** out) {
+    static std::mutex mu;
+    static unsigned int* addr[64] = {nullptr};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FP8_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return FP8_ERR_CUDA;
+        addr[dev] = reinterpret_cast<unsigned int*>(p);
+    }
+    *out = addr[dev];
+    return FP8_OK;
+}
+
+fp8_status fp8_quantize_current_static(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o, uint8_t* out,
+                                       float* amax_dev, float* scale_dev, float* scale_inv_dev, void* stream) {
+    if (!amax_dev || !scale_dev || !scale_inv_dev || ((!x || !out) && n)) return FP8_ERR_NULL;
+    if ((t != FP8_F32 && t != FP8_BF16) || (f != FP8_E4M3 && f != FP8_E5M2) || (o != FP8_SATURATE && o != FP8_NOSAT))
+        return FP8_ERR_ENUM;
+    if (n > FP8_STATIC_MAX_ELEMENTS) return FP8_ERR_UNSUPPORTED;
+    unsigned int* scratch = nullptr;
+    fp8_status s = static_scratch_address(&scratch);
+    if (s != FP8_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the last call left (zeros, unless that call gave up on its barrier): start clean
+    if (cudaMemsetAsync(scratch, 0, 16, st) != cudaSuccess) return FP8_ERR_CUDA;
+    count_launches(1);
+    return fp8b200::launch_quantize_current(x, t, n, f, o, out, amax_dev, scale_dev, scale_inv_dev, scratch, st);
+}
+
+
 void fp8_cast_read_clear_latch(unsigned int out2[2]) {
     out2[0] = out2[1] = 0u;
     if (cudaMemcpyFromSymbol(out2, fp8b200::g_cast_latch, 2 * sizeof(unsigned int)) != cudaSuccess) return;
