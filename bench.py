@@ -35,6 +35,10 @@ UNIT = "TFLOP/s"
 WORKLOAD = ("transformer linear layer fwd+bwd, hidden 4096->16384, 8192 tokens: amax+scale+quantize of X,W (E4M3) and dY (E5M2), "
             "one dequantize, fprop/dgrad/wgrad FP8 GEMMs, bf16 out + epilogue amax")
 TOKENS, D_IN, D_OUT, W_SIGMA = 8192, 4096, 16384, 0.02
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (same workload):
+# forward GEMM 168.5 MB + 225.5 MB; one-launch conversion, mean of the X, W and dY launches.
+NCU_TRAFFIC_GEMM_BYTES = 3.94e8
+NCU_TRAFFIC_QUANTIZE_CURRENT_BYTES = 2.68e8
 NOMINAL_FP8_TFLOPS = 4500.0
 NOMINAL_HBM_GBS = 8000.0
 
@@ -408,7 +412,8 @@ def run_ours(args):
         achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12
         fp8_peak = 2.0 * pk["bf16_sustained"]            # fp8 : bf16 nominal ratio is 2
         roofline = {"bound": "tensor", "kernel": "k_gemm_fp8", "achieved": round(achieved, 1), "peak": round(fp8_peak, 1),
-                    "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4), "traffic": None,
+                    "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4), "traffic": NCU_TRAFFIC_GEMM_BYTES,
+                    "traffic_note": "DRAM bytes per launch, ncu capture of the forward GEMM (profiles/gemm_fp8_forward_hidden4096.md); algorithmic 3.69e8",
                     "peak_source": "2 x %s bf16 sustained cuBLAS TFLOP/s (fp8:bf16 nominal ratio)" % pk["source"],
                     "frac_of_nominal_4500": round(achieved / NOMINAL_FP8_TFLOPS, 4),
                     "per_gemm_tflops": {k: round(gemm_flops / (avg[k] * 1e-3) / 1e12, 1) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}}
@@ -418,7 +423,8 @@ def run_ours(args):
         cast_gbs = step.cast_bytes / (cast_ms * 1e-3) / 1e9
         n_x = TOKENS * D_IN + D_IN * D_OUT + TOKENS * D_OUT
         roofline_cast = {"bound": "hbm", "kernel": "casts of the step: " + " + ".join(cast_labels), "achieved": round(cast_gbs, 1),
-                         "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": round(cast_gbs / pk["hbm_gbs"], 4), "traffic": None,
+                         "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": round(cast_gbs / pk["hbm_gbs"], 4),
+                         "traffic": NCU_TRAFFIC_QUANTIZE_CURRENT_BYTES if "quantize_current" in avg else None,
                          "peak_source": pk["source"] + " copy bandwidth", "frac_of_nominal_8000": round(cast_gbs / NOMINAL_HBM_GBS, 4),
                          "algorithmic_bytes": "5 B per bf16 element for amax+quantize (two reads, one write), 3 B per element for dequantize; "
                                               "re-reads served by L2 still count as algorithmic bytes"}
