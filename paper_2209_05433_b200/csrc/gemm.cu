@@ -291,9 +291,10 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
     const int worker = blockIdx.x / CG, num_workers = gridDim.x / CG;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int k_blocks = (int)((p.K + BK - 1) / BK);
+    const int k_pad = (k_blocks + 1) & ~1;                        // K-blocks are consumed two at a time
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), CG); mbar_init(smem_u32(&bars->empty[s]), 1); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), 2 * CG); mbar_init(smem_u32(&bars->empty[s]), 1); }
         for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(smem_u32(&bars->acc_full[a]), 1); mbar_init(smem_u32(&bars->acc_empty[a]), EPI_WARPS * CG); }
         bars->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -324,7 +325,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
             const int m0 = tm * G::TILE_M + (int)cta_rank * BM;                 // this CTA's 128 rows of A
             const int n0 = tn * BN + (int)cta_rank * (BN / CG);                 // this CTA's rows of B
-            for (int kb = 0; kb < k_blocks; ++kb) {
+            for (int kb = 0; kb < k_pad; ++kb) {
                 PROF_BEGIN
                 ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, WAIT_EMPTY);
                 PROF_END(prof_acc0)
@@ -333,23 +334,31 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     const uint32_t sa = ring + stage * STAGE_BYTES;
                     const uint32_t sb = sa + A_BYTES;
                     const int k0 = kb * BK;
+                    const uint32_t pair_bar = smem_u32(&bars->full[stage >> 1]);          // one barrier per two stages
                     if (CG == 2) {
-                        const uint32_t full = map_to_cta(smem_u32(&bars->full[stage]), 0);   // the leader's barrier
-                        mbar_arrive_expect_tx_cluster(full, STAGE_BYTES);
-                        if (A_MN) tma_load_2d_pair(sa, &map_a, m0, k0, full, keep);     // box {128 m, 128 k}
-                        else      tma_load_2d_pair(sa, &map_a, k0, m0, full, keep);     // box {128 k, 128 m}
-                        if (B_MN) tma_load_2d_pair(sb, &map_b, n0, k0, full, keep);     // box {128 n, 128 k}
-                        else      tma_load_2d_pair(sb, &map_b, k0, n0, full, keep);     // box {128 k, 128 n}
-                    } else {
-                        const uint32_t full = smem_u32(&bars->full[stage]);
-                        mbar_arrive_expect_tx(full, STAGE_BYTES);
-                        if (A_MN) tma_load_2d(sa, &map_a, m0, k0, full, keep);
-                        else      tma_load_2d(sa, &map_a, k0, m0, full, keep);
-                        if (B_MN) {                                               // two boxes {128 n, 128 k}
-                            tma_load_2d(sb, &map_b, n0, k0, full, keep);
-                            tma_load_2d(sb + G::B_BYTES / 2, &map_b, n0 + 128, k0, full, keep);
+                        const uint32_t full = map_to_cta(pair_bar, 0);                    // the leader's barrier
+                        if (kb < k_blocks) {
+                            mbar_arrive_expect_tx_cluster(full, STAGE_BYTES);
+                            if (A_MN) tma_load_2d_pair(sa, &map_a, m0, k0, full, keep);     // box {128 m, 128 k}
+                            else      tma_load_2d_pair(sa, &map_a, k0, m0, full, keep);     // box {128 k, 128 m}
+                            if (B_MN) tma_load_2d_pair(sb, &map_b, n0, k0, full, keep);     // box {128 n, 128 k}
+                            else      tma_load_2d_pair(sb, &map_b, k0, n0, full, keep);     // box {128 k, 128 n}
                         } else {
-                            tma_load_2d(sb, &map_b, k0, n0, full, keep);                // box {128 k, 256 n}
+                            mbar_arrive_cluster(full);                                    // padding block: nothing to load
+                        }
+                    } else {
+                        if (kb < k_blocks) {
+                            mbar_arrive_expect_tx(pair_bar, STAGE_BYTES);
+                            if (A_MN) tma_load_2d(sa, &map_a, m0, k0, pair_bar, keep);
+                            else      tma_load_2d(sa, &map_a, k0, m0, pair_bar, keep);
+                            if (B_MN) {                                               // two boxes {128 n, 128 k}
+                                tma_load_2d(sb, &map_b, n0, k0, pair_bar, keep);
+                                tma_load_2d(sb + G::B_BYTES / 2, &map_b, n0 + 128, k0, pair_bar, keep);
+                            } else {
+                                tma_load_2d(sb, &map_b, k0, n0, pair_bar, keep);        // box {128 k, 256 n}
+                            }
+                        } else {
+                            mbar_arrive(pair_bar);
                         }
                     }
                 }
@@ -372,37 +381,46 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             if (!ok) break;
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * BN;
-            for (int kb = 0; kb < k_blocks; ++kb) {
+            for (int kb = 0; kb < k_pad; kb += 2) {
+                // one wait per TWO K-blocks: every barrier query between MMA issues costs about one MMA time
                 PROF_BEGIN
-                ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, WAIT_FULL);
+                ok = mbar_wait(smem_u32(&bars->full[stage >> 1]), phase, abort_flag, WAIT_FULL);
                 PROF_END(prof_acc0)
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t sa = ring + stage * STAGE_BYTES;
-                    const uint32_t sb = sa + A_BYTES;
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // K-major: 8-row groups 1024 B apart, +32 B per K step inside the swizzled row.
-                        // MN-major: 8-k groups 1024 B apart, 128-wide MN blocks BK*128 B apart, +32 k-rows per step.
-                        const uint64_t da = A_MN ? smem_desc(sa + k * UMMA_K * 128, BK * 128, 1024)
-                                                 : smem_desc(sa + k * UMMA_K, 16, 1024);
-                        const uint64_t db = B_MN ? smem_desc(sb + k * UMMA_K * 128, BK * 128, 1024)
-                                                 : smem_desc(sb + k * UMMA_K, 16, 1024);
-                        if (CG == 2) tc_mma_f8_pair(tmem_d, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
-                        else         tc_mma_f8(tmem_d, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
-                    }
-                    // frees the smem stage (in both CTAs) when the MMAs retire; the last block also publishes the accumulator
-                    if (CG == 2) {
-                        tc_commit_pair(smem_u32(&bars->empty[stage]));
-                        if (kb == k_blocks - 1) tc_commit_pair(smem_u32(&bars->acc_full[acc]));
-                    } else {
-                        tc_commit(smem_u32(&bars->empty[stage]));
-                        if (kb == k_blocks - 1) tc_commit(smem_u32(&bars->acc_full[acc]));
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t st = stage + h;
+                        if (kb + h < k_blocks) {
+                            const uint32_t sa = ring + st * STAGE_BYTES;
+                            const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+                            for (int k = 0; k < BK / UMMA_K; ++k) {
+                                // K-major: 8-row groups 1024 B apart, +32 B per K step inside the swizzled row.
+                                // MN-major: 8-k groups 1024 B apart, 128-wide MN blocks BK*128 B apart, +32 k-rows per step.
+                                const uint64_t da = A_MN ? smem_desc(sa + k * UMMA_K * 128, BK * 128, 1024)
+                                                         : smem_desc(sa + k * UMMA_K, 16, 1024);
+                                const uint64_t db = B_MN ? smem_desc(sb + k * UMMA_K * 128, BK * 128, 1024)
+                                                         : smem_desc(sb + k * UMMA_K, 16, 1024);
+                                if (CG == 2) tc_mma_f8_pair(tmem_d, da, db, p.idesc, (kb | h | k) != 0 ? 1u : 0u);
+                                else         tc_mma_f8(tmem_d, da, db, p.idesc, (kb | h | k) != 0 ? 1u : 0u);
+                            }
+                        }
+                        // frees the smem stage (in both CTAs) when the MMAs retire (a padding block frees at once);
+                        // the last real block also publishes the accumulator
+                        if (CG == 2) {
+                            tc_commit_pair(smem_u32(&bars->empty[st]));
+                            if (kb + h == k_blocks - 1) tc_commit_pair(smem_u32(&bars->acc_full[acc]));
+                        } else {
+                            tc_commit(smem_u32(&bars->empty[st]));
+                            if (kb + h == k_blocks - 1) tc_commit(smem_u32(&bars->acc_full[acc]));
+                        }
                     }
                 }
                 __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                stage += 2;
+                if (stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
         PROF_STORE(3, 4, 5)
