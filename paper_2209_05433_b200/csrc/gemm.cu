@@ -71,6 +71,7 @@ template <int CG> struct Geo {
     static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = CG == 1 ? 4 : 6;
     static constexpr int TILE_M = BM * CG;
+    static constexpr int FG = 2;                                    // K-blocks (stages) consumed per full-barrier wait
 };
 constexpr uint32_t SMEM_TILES = 4 * (A_BYTES + BN * BK);            // = 6 * (A_BYTES + BN/2 * BK)
 constexpr uint32_t EPI_BUF_BYTES = 4096;                            // 32 rows x 128 B, one TMA store box
@@ -291,10 +292,11 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
     const int worker = blockIdx.x / CG, num_workers = gridDim.x / CG;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int k_blocks = (int)((p.K + BK - 1) / BK);
-    const int k_pad = (k_blocks + 1) & ~1;                        // K-blocks are consumed two at a time
+    constexpr int FG = G::FG;
+    const int k_pad = (k_blocks + FG - 1) / FG * FG;               // K-blocks are consumed FG at a time
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), 2 * CG); mbar_init(smem_u32(&bars->empty[s]), 1); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), FG * CG); mbar_init(smem_u32(&bars->empty[s]), 1); }
         for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(smem_u32(&bars->acc_full[a]), 1); mbar_init(smem_u32(&bars->acc_empty[a]), EPI_WARPS * CG); }
         bars->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -334,7 +336,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     const uint32_t sa = ring + stage * STAGE_BYTES;
                     const uint32_t sb = sa + A_BYTES;
                     const int k0 = kb * BK;
-                    const uint32_t pair_bar = smem_u32(&bars->full[stage >> 1]);          // one barrier per two stages
+                    const uint32_t pair_bar = smem_u32(&bars->full[stage / FG]);          // one barrier per FG stages
                     if (CG == 2) {
                         const uint32_t full = map_to_cta(pair_bar, 0);                    // the leader's barrier
                         if (kb < k_blocks) {
@@ -381,16 +383,16 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             if (!ok) break;
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * BN;
-            for (int kb = 0; kb < k_pad; kb += 2) {
+            for (int kb = 0; kb < k_pad; kb += FG) {
                 // one wait per TWO K-blocks: every barrier query between MMA issues costs about one MMA time
                 PROF_BEGIN
-                ok = mbar_wait(smem_u32(&bars->full[stage >> 1]), phase, abort_flag, WAIT_FULL);
+                ok = mbar_wait(smem_u32(&bars->full[stage / FG]), phase, abort_flag, WAIT_FULL);
                 PROF_END(prof_acc0)
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
+                    for (int h = 0; h < FG; ++h) {
                         const uint32_t st = stage + h;
                         if (kb + h < k_blocks) {
                             const uint32_t sa = ring + st * STAGE_BYTES;
@@ -419,7 +421,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     }
                 }
                 __syncwarp();
-                stage += 2;
+                stage += FG;
                 if (stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
