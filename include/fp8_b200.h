@@ -154,6 +154,26 @@ fp8_status fp8_dequantize(const uint8_t* c, size_t n, fp8_format f,
                           const float* scale_inv_dev, void* out, fp8_wide t, void* stream);
 
 /*
+ * fp8_fake_quantize — Section 4: the paper's own experiments ran "simulated FP8": tensors were converted
+ * to FP8 (scale factor, rounding and saturation included) and straight back to the wider type, and the
+ * arithmetic stayed in that wider type.  This is that round trip in one pass over the tensor:
+ *   out_i = round_t( decode_f( encode_f( binary32(x_i) * scale ) ) * scale_inv ),  out has the type of x.
+ * Bit for bit the composition of fp8_quantize and fp8_dequantize, without the intermediate code tensor
+ * (4 B per bf16 element of traffic instead of 6).
+ */
+fp8_status fp8_fake_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o,
+                             const float* scale_dev, const float* scale_inv_dev, void* out, void* stream);
+
+/*
+ * fp8_scale_pow2_from_amax — Section 3.2: a programmable exponent bias "is equivalent to allowing only
+ * powers of 2 as scaling factors".  scale = the largest power of two not above fmax/amax (same guards
+ * as fp8_scale_from_amax), scale_inv = 1/scale (exact).  Converting with this scale is converting to an
+ * E4M3/E5M2 variant whose exponent bias is shifted by log2(scale) (the bias sweep of Section 4.3).
+ */
+fp8_status fp8_scale_pow2_from_amax(const float* amax_dev, fp8_format f,
+                                    float* scale_dev, float* scale_inv_dev, void* stream);
+
+/*
  * fp8_gemm — Sections 2, 3 and 4.1: the matrix multiply on FP8 inputs with a
  * higher-precision result, unscaled once per dot product.
  *   D[i,j] = round_out( (sum_k decode_fa(A[i,k]) * decode_fb(B[k,j])) * (sa_inv * sb_inv) )

@@ -77,6 +77,8 @@ def _load():
     lib.fp8o_amax_bf16.argtypes = [u16p, c.c_size_t]
     lib.fp8o_scale_from_amax.restype = None
     lib.fp8o_scale_from_amax.argtypes = [c.c_float, c.c_int, f32p, f32p]
+    lib.fp8o_scale_pow2_from_amax.restype = None
+    lib.fp8o_scale_pow2_from_amax.argtypes = [c.c_float, c.c_int, f32p, f32p]
     gemm_common = [u8p, c.c_int, c.c_int64, c.c_int64, u8p, c.c_int, c.c_int64, c.c_int64]
     lib.fp8o_gemm_rows.restype = None
     lib.fp8o_gemm_rows.argtypes = gemm_common + [c.c_int64, c.c_int64, c.c_int64, c.c_int64,
@@ -139,6 +141,18 @@ def scale_from_amax(amax, fmt: int):
     s, si = ctypes.c_float(), ctypes.c_float()
     _load().fp8o_scale_from_amax(ctypes.c_float(np.float32(amax)), fmt, ctypes.byref(s), ctypes.byref(si))
     return np.float32(s.value), np.float32(si.value)
+
+
+def scale_pow2_from_amax(amax, fmt: int):
+    s, si = ctypes.c_float(), ctypes.c_float()
+    _load().fp8o_scale_pow2_from_amax(ctypes.c_float(np.float32(amax)), fmt, ctypes.byref(s), ctypes.byref(si))
+    return np.float32(s.value), np.float32(si.value)
+
+
+def fake_quantize(x: np.ndarray, scale, scale_inv, fmt: int, overflow: int = SATURATE, threads: int = 1) -> np.ndarray:
+    """Simulated FP8 (Section 4): convert to FP8 and straight back, in the type of x."""
+    wide = "f32" if _wide_kind(np.ascontiguousarray(x).reshape(-1)) == "f32" else "bf16"
+    return dequantize(quantize(x, scale, fmt, overflow, threads), scale_inv, fmt, wide, threads)
 
 
 # ------------------------------------------------------------------ tensors --

@@ -269,6 +269,20 @@ void fp8o_scale_from_amax(float amax, int fmt, float* scale, float* scale_inv)
     *scale_inv = (float)(1.0 / (double)s);
 }
 
+/* Section 3.2: a programmable exponent bias is the same as a power-of-two scale
+ * factor.  The scale is the largest power of two not above fmax / amax (the
+ * quotient with the guards of fp8o_scale_from_amax); its inverse is exact. */
+void fp8o_scale_pow2_from_amax(float amax, int fmt, float* scale, float* scale_inv)
+{
+    float s0, unused;
+    fp8o_scale_from_amax(amax, fmt, &s0, &unused);
+    int e;
+    (void)frexp((double)s0, &e);                 /* s0 = m * 2^e, m in [0.5, 1)  ->  2^(e-1) <= s0 < 2^e */
+    float s = (float)ldexp(1.0, e - 1);          /* exact, also for subnormal s0 */
+    *scale = s;
+    *scale_inv = (float)(1.0 / (double)s);
+}
+
 /* --------------------------------------------------------------------- GEMM */
 
 /* One output element of D = (A.B) * sa_inv * sb_inv.

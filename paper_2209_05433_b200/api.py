@@ -20,7 +20,8 @@ SATURATE, NOSAT = 0, 1       # fp8_overflow
 MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
 
 EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
-           "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_gemm",
+           "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_fake_quantize",
+           "fp8_scale_pow2_from_amax", "fp8_gemm",
            "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
 
 
@@ -71,6 +72,10 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_quantize_current_static.argtypes = [vp, i32, sz, i32, i32, vp, vp, vp, vp, vp]
     lib.fp8_dequantize.restype = i32
     lib.fp8_dequantize.argtypes = [vp, sz, i32, vp, vp, i32, vp]
+    lib.fp8_fake_quantize.restype = i32
+    lib.fp8_fake_quantize.argtypes = [vp, i32, sz, i32, i32, vp, vp, vp, vp]
+    lib.fp8_scale_pow2_from_amax.restype = i32
+    lib.fp8_scale_pow2_from_amax.argtypes = [vp, i32, vp, vp, vp]
     lib.fp8_gemm.restype = i32
     lib.fp8_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.fp8_async_status.restype = i32
@@ -177,6 +182,19 @@ def fp8_dequantize(codes: torch.Tensor, fmt: int, scale_inv: torch.Tensor, out: 
         raise TypeError("codes must be uint8 and out must have as many elements")
     _check(load().fp8_dequantize(_dev(codes, "codes"), codes.numel(), fmt, _scalar(scale_inv, "scale_inv"),
                                  _dev(out, "out"), _wide_of(out), _stream()), "fp8_dequantize")
+
+
+def fp8_fake_quantize(x: torch.Tensor, fmt: int, scale: torch.Tensor, scale_inv: torch.Tensor, out: torch.Tensor,
+                      overflow: int = SATURATE) -> None:
+    if out.dtype != x.dtype or out.numel() != x.numel():
+        raise TypeError("out must have the dtype and size of x")
+    _check(load().fp8_fake_quantize(_dev(x, "x"), _wide_of(x), x.numel(), fmt, overflow, _scalar(scale, "scale"),
+                                    _scalar(scale_inv, "scale_inv"), _dev(out, "out"), _stream()), "fp8_fake_quantize")
+
+
+def fp8_scale_pow2_from_amax(amax: torch.Tensor, fmt: int, scale_out: torch.Tensor, scale_inv_out: torch.Tensor) -> None:
+    _check(load().fp8_scale_pow2_from_amax(_scalar(amax, "amax"), fmt, _scalar(scale_out, "scale_out"),
+                                           _scalar(scale_inv_out, "scale_inv_out"), _stream()), "fp8_scale_pow2_from_amax")
 
 
 def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,

@@ -516,6 +516,95 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
 }
 
 // ---------------------------------------------------------------------------
+// fake quantization: wide -> FP8 -> wide in one pass (what "simulated FP8" runs, Section 4)
+// ---------------------------------------------------------------------------
+
+// one scaled value -> its FP8 code -> back to binary32 times scale_inv (scalar path, any input)
+template <int FMT, bool NOSAT>
+__device__ __forceinline__ float fake_one(float xf, float scale, float scale_inv) {
+    const uint32_t code = encode_scaled<FMT, NOSAT>(xf * scale, __float_as_uint(xf));
+    return decode_pair<FMT>(code).x * scale_inv;
+}
+
+template <int WIDE, int FMT, bool NOSAT, int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+k_fake_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale_dev,
+                const float* __restrict__ scale_inv_dev, void* __restrict__ out) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    const float scale = *scale_dev, si = *scale_inv_dev;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    const size_t n_items = n / EPI;
+    const size_t per_chunk = (size_t)kThreads * UNROLL;
+    const size_t n_chunks = (n_items + per_chunk - 1) / per_chunk;
+
+    auto emit = [&](size_t i, const uint4& v) {
+        if (WIDE == kWideBF16) {
+            const uint2 c = quantize_item_bf16<FMT, NOSAT>(v, scale);
+            const float2 a = decode_pair<FMT>(c.x), b = decode_pair<FMT>(c.x >> 16);
+            const float2 d = decode_pair<FMT>(c.y), e = decode_pair<FMT>(c.y >> 16);
+            uint4 o;
+            o.x = pack_bf16(a.x * si, a.y * si);
+            o.y = pack_bf16(b.x * si, b.y * si);
+            o.z = pack_bf16(d.x * si, d.y * si);
+            o.w = pack_bf16(e.x * si, e.y * si);
+            st_out(reinterpret_cast<uint4*>(out) + i, o);
+        } else {
+            const uint32_t c = quantize_item_f32<FMT, NOSAT>(v, scale);
+            const float2 a = decode_pair<FMT>(c), b = decode_pair<FMT>(c >> 16);
+            st_out(reinterpret_cast<float4*>(out) + i, make_float4(a.x * si, a.y * si, b.x * si, b.y * si));
+        }
+    };
+
+    for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        const size_t base = chunk * per_chunk + threadIdx.x;
+        if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
+            uint4 v[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) emit(base + (size_t)u * kThreads, v[u]);
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const size_t i = base + (size_t)u * kThreads;
+                if (i < n_items) emit(i, ld_nc_v4(xv + i));
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < n - n_items * EPI) {    // ragged tail
+        const size_t i = n_items * EPI + threadIdx.x;
+        const float v = fake_one<FMT, NOSAT>(scalar_load<WIDE>(x, i), scale, si);
+        if (WIDE == kWideBF16) reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)pack_bf16(v, 0.0f);
+        else                   reinterpret_cast<float*>(out)[i] = v;
+    }
+}
+
+template <int WIDE, int FMT, bool NOSAT>
+__global__ void __launch_bounds__(kThreads)
+k_fake_quantize_elementwise(const void* __restrict__ x, size_t n, const float* __restrict__ scale_dev,
+                            const float* __restrict__ scale_inv_dev, void* __restrict__ out) {
+    const float scale = *scale_dev, si = *scale_inv_dev;
+    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (size_t)gridDim.x * kThreads) {
+        const float v = fake_one<FMT, NOSAT>(scalar_load<WIDE>(x, i), scale, si);
+        if (WIDE == kWideBF16) reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)pack_bf16(v, 0.0f);
+        else                   reinterpret_cast<float*>(out)[i] = v;
+    }
+}
+
+// power-of-two scale: the largest power of two not above fmax / amax (same guards as k_scale_from_amax).
+// With such a scale the conversion is the paper's "programmable exponent bias" variant (Section 3.2).
+__global__ void k_scale_pow2_from_amax(const float* amax_dev, float fmax, float* scale_dev, float* scale_inv_dev) {
+    float s, si;
+    scale_pair_from_amax(*amax_dev, fmax, s, si);
+    uint32_t b = __float_as_uint(s);
+    if ((b >> 23) != 0u) b &= 0x7F800000u;                       // normal: drop the fraction
+    else if (b != 0u) b = 1u << (31 - __clz(b));                  // subnormal: keep the leading bit
+    s = __uint_as_float(b);
+    *scale_dev = s;
+    *scale_inv_dev = __fdiv_rn(1.0f, s);
+}
+
+// ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
 
@@ -646,6 +735,23 @@ fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_form
                  : launch_current<kWideBF16, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
 }
 
+template <int WIDE, int FMT, bool NOSAT>
+static fp8_status launch_fake(const void* x, size_t n, const float* scale, const float* si, void* out, cudaStream_t st) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int UNROLL = 2;
+    if (aligned16(x) && aligned16(out)) {
+        auto k = k_fake_quantize<WIDE, FMT, NOSAT, UNROLL>;
+        const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL));
+        k<<<grid, kThreads, 0, st>>>(x, n, scale, si, out);
+    } else {
+        auto k = k_fake_quantize_elementwise<WIDE, FMT, NOSAT>;
+        const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
+        k<<<grid, kThreads, 0, st>>>(x, n, scale, si, out);
+    }
+    count_launches(1);
+    return launch_status();
+}
+
 }  // namespace fp8b200
 
 using namespace fp8b200;
@@ -749,6 +855,34 @@ void fp8_cast_read_clear_latch(unsigned int out2[2]) {
         const unsigned int zero[2] = {0u, 0u};
         cudaMemcpyToSymbol(fp8b200::g_cast_latch, zero, sizeof(zero));
     }
+}
+
+fp8_status fp8_fake_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o,
+                             const float* scale_dev, const float* scale_inv_dev, void* out, void* stream) {
+    if (!scale_dev || !scale_inv_dev || ((!x || !out) && n)) return FP8_ERR_NULL;
+    if ((t != FP8_F32 && t != FP8_BF16) || (f != FP8_E4M3 && f != FP8_E5M2) || (o != FP8_SATURATE && o != FP8_NOSAT))
+        return FP8_ERR_ENUM;
+    if (n == 0) return FP8_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool nosat = o == FP8_NOSAT;
+    if (t == FP8_F32) {
+        if (f == FP8_E4M3) return nosat ? launch_fake<kWideF32, kE4M3, true>(x, n, scale_dev, scale_inv_dev, out, st)
+                                        : launch_fake<kWideF32, kE4M3, false>(x, n, scale_dev, scale_inv_dev, out, st);
+        return nosat ? launch_fake<kWideF32, kE5M2, true>(x, n, scale_dev, scale_inv_dev, out, st)
+                     : launch_fake<kWideF32, kE5M2, false>(x, n, scale_dev, scale_inv_dev, out, st);
+    }
+    if (f == FP8_E4M3) return nosat ? launch_fake<kWideBF16, kE4M3, true>(x, n, scale_dev, scale_inv_dev, out, st)
+                                    : launch_fake<kWideBF16, kE4M3, false>(x, n, scale_dev, scale_inv_dev, out, st);
+    return nosat ? launch_fake<kWideBF16, kE5M2, true>(x, n, scale_dev, scale_inv_dev, out, st)
+                 : launch_fake<kWideBF16, kE5M2, false>(x, n, scale_dev, scale_inv_dev, out, st);
+}
+
+fp8_status fp8_scale_pow2_from_amax(const float* amax_dev, fp8_format f, float* scale_dev, float* scale_inv_dev, void* stream) {
+    if (!amax_dev || !scale_dev || !scale_inv_dev) return FP8_ERR_NULL;
+    if (f != FP8_E4M3 && f != FP8_E5M2) return FP8_ERR_ENUM;
+    k_scale_pow2_from_amax<<<1, 1, 0, (cudaStream_t)stream>>>(amax_dev, f == FP8_E4M3 ? 448.0f : 57344.0f, scale_dev, scale_inv_dev);
+    count_launches(1);
+    return launch_status();
 }
 
 fp8_status fp8_dequantize(const uint8_t* c, size_t n, fp8_format f, const float* scale_inv_dev, void* out, fp8_wide t, void* stream) {

@@ -297,3 +297,48 @@ def test_quantize_current_specials_and_unaligned():
         ws, wsi = oracle.scale_from_amax(np.array([want_bits], dtype=np.uint32).view(np.float32)[0], oracle.E4M3)
         assert a.cpu().numpy().view(np.uint32)[0] == want_bits and s.item() == ws and si.item() == wsi
         _assert_codes(out.cpu().numpy(), oracle.quantize(x_np, ws, oracle.E4M3), x_np)
+
+
+# ------------------------------- simulated FP8 round trip and power-of-two scale --
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_scale_pow2_from_amax(fmt):
+    rng = np.random.default_rng(18)
+    vals = np.concatenate([np.exp2(rng.uniform(-140, 127, size=300)), [0.0, np.inf, np.nan, 1.0, 448.0, 57344.0, 1e-44, 3.4e38]]).astype(np.float32)
+    s, si = _scalar(0.0), _scalar(0.0)
+    for v in vals:
+        api.fp8_scale_pow2_from_amax(_scalar(float(v)), fmt, s, si)
+        ws, wsi = oracle.scale_pow2_from_amax(v, fmt)
+        assert s.cpu().numpy().view(np.uint32)[0] == np.array([ws]).view(np.uint32)[0], v
+        assert si.cpu().numpy().view(np.uint32)[0] == np.array([wsi]).view(np.uint32)[0], v
+
+
+@pytest.mark.parametrize("wide,name", [(torch.float32, "f32"), (torch.bfloat16, "bf16")])
+@pytest.mark.parametrize("fmt", FMTS)
+def test_fake_quantize_equals_quantize_then_dequantize(wide, name, fmt):
+    for n, off in ((0, 0), (5, 0), (4099, 0), ((1 << 20) + 7, 0), (70001, 3)):
+        base = synth.normal_laplace_mixture(n + 16, 11, synth.T_ID, dtype=wide, device=DEV)
+        x = base[off: off + n]
+        if n > 100:
+            x = x.clone() if off == 0 else x
+            x[7] = float("nan"); x[8] = float("-inf"); x[9] = 1e30
+        x_np = to_np_bits(x)
+        for overflow in (api.SATURATE, api.NOSAT):
+            for scale, scale_inv in ((3.0, 1.0 / 3.0), (0.25, 4.0)):
+                out = torch.zeros(n + 16, dtype=wide, device=DEV)
+                api.fp8_fake_quantize(x, fmt, _scalar(scale), _scalar(scale_inv), out[off: off + n] if off else out[:n], overflow)
+                torch.cuda.synchronize()
+                got = to_np_bits(out[off: off + n] if off else out[:n])
+                want = oracle.fake_quantize(x_np, np.float32(scale), np.float32(scale_inv), fmt, overflow, threads=THREADS)
+                ok = same_with_nan(got, want, name)
+                assert ok.all(), (n, off, overflow, scale, np.nonzero(~ok)[0][:5])
+
+
+def test_fake_quantize_every_bf16_value():
+    x = _all_bf16().to(DEV)
+    xb = to_np_bits(x)
+    for fmt in FMTS:
+        out = torch.empty_like(x)
+        api.fp8_fake_quantize(x, fmt, _scalar(0.37), _scalar(1.0 / 0.37), out)
+        want = oracle.fake_quantize(xb, np.float32(0.37), np.float32(1.0 / 0.37), fmt)
+        assert same_with_nan(to_np_bits(out), want, "bf16").all()

@@ -374,6 +374,40 @@ def test_scale_from_amax(fmt, maxcode):
     assert s == np.finfo(np.float32).max and np.isfinite(si)
 
 
+@pytest.mark.parametrize("fmt,maxcode", [(E4M3, 0x7E), (E5M2, 0x7B)])
+def test_power_of_two_scale_from_amax(fmt, maxcode):
+    fmax = oracle.FMT_MAX[fmt]
+    rng = np.random.default_rng(21)
+    for a in np.concatenate([np.exp2(rng.uniform(-100, 100, size=1000)), [1.0, 448.0, 57344.0, 3.7, 7.0, 0.875]]).astype(np.float32):
+        s, si = oracle.scale_pow2_from_amax(a, fmt)
+        s0 = np.float32(fmax) / a
+        m, e = np.frexp(np.float64(s))
+        assert m == 0.5                                   # a power of two
+        assert s <= s0 < 2 * np.float64(s)                # the largest one not above fmax / amax
+        assert np.float64(s) * np.float64(si) == 1.0      # the inverse is exact
+        # the scaled maximum lands in the top binade of the format and never overflows
+        code = oracle.encode(a * s, fmt, NOSAT)
+        assert code <= maxcode and oracle.decode(code, fmt) > fmax / 2 * (1 - 2.0 ** -3)
+    for a in (0.0, np.nan, np.inf):
+        assert oracle.scale_pow2_from_amax(np.float32(a), fmt) == (1.0, 1.0)
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2])
+def test_fake_quantize_values_are_representable_and_fixed_points(fmt):
+    # simulated FP8 (Section 4): the result is the nearest representable value times 1/scale,
+    # and applying it twice changes nothing when the scale is a power of two
+    rng = np.random.default_rng(22)
+    x = (rng.standard_normal(1 << 14) * 3).astype(np.float32)
+    s, si = oracle.scale_pow2_from_amax(np.abs(x).max(), fmt)
+    y = oracle.fake_quantize(x, s, si, fmt)
+    t = oracle.decode_table(fmt)
+    finite = t[np.isfinite(t)]
+    assert np.isin(y.astype(np.float64) * float(s), finite).all()
+    assert np.array_equal(oracle.fake_quantize(y, s, si, fmt), y)
+    near = finite[np.abs(finite[None, :] - (x.astype(np.float64) * float(s))[:, None]).argmin(axis=1)]
+    assert np.all(np.abs(y.astype(np.float64) * float(s) - x.astype(np.float64) * float(s)) <= np.abs(near - x.astype(np.float64) * float(s)) + 1e-300)
+
+
 # ------------------------------------------------------------ bf16 rounding --
 
 def test_f64_to_bf16_single_rounding():
