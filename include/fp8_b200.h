@@ -207,6 +207,24 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
                     float* amax_d_dev, void* stream);
 
 /*
+ * fp8_gemm_fp8out — Section 2: operations on FP8 inputs produce higher-precision results, "optionally
+ * converting the results to FP8 prior to writing them to memory".  Same contraction as fp8_gemm, but the
+ * epilogue converts instead of storing a wide value:
+ *   v[i,j] = (sum_k decode_fa(A[i,k]) * decode_fb(B[k,j])) * (sa_inv * sb_inv)      (binary32)
+ *   D[i,j] = encode_fd( v[i,j] * scale_d )       conversion rules of fp8_quantize (RNE, specials, `od`)
+ *   *amax_d_dev = amax over v, i.e. BEFORE the output scale and the conversion: it is the quantity the
+ *                 next scale factor for this tensor is chosen from (scale_d itself comes from an earlier
+ *                 step, as the scale-history recipes the paper leaves to software do).
+ *   D            M x N codes, D[i,j] at D[i*ldd + j]; d->out is ignored; D and ldd 16-byte aligned.
+ *   scale_d_dev  device float.
+ * Everything else (operands, layouts, alignment, edge cases) as fp8_gemm.
+ */
+fp8_status fp8_gemm_fp8out(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, uint8_t* D,
+                           fp8_format fd, fp8_overflow od,
+                           const float* scale_inv_a_dev, const float* scale_inv_b_dev, const float* scale_d_dev,
+                           float* amax_d_dev, void* stream);
+
+/*
  * fp8_async_status — reads and clears the device-side error latch of the
  * current device (synchronises the device).  FP8_OK, or FP8_ERR_TIMEOUT if a
  * kernel gave up on a bounded wait since the last call; *detail (optional, host

@@ -21,7 +21,7 @@ MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
 
 EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
            "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_fake_quantize",
-           "fp8_scale_pow2_from_amax", "fp8_gemm",
+           "fp8_scale_pow2_from_amax", "fp8_gemm", "fp8_gemm_fp8out",
            "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
 
 
@@ -78,6 +78,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_scale_pow2_from_amax.argtypes = [vp, i32, vp, vp, vp]
     lib.fp8_gemm.restype = i32
     lib.fp8_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp]
+    lib.fp8_gemm_fp8out.restype = i32
+    lib.fp8_gemm_fp8out.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
     lib.fp8_async_status.restype = i32
     lib.fp8_async_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
     lib.fp8_status_string.restype = ctypes.c_char_p
@@ -217,6 +219,27 @@ def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: in
     _check(load().fp8_gemm(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
                            _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
                            None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()), "fp8_gemm")
+
+
+def fp8_gemm_fp8out(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor, fd: int,
+                    scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, scale_d: torch.Tensor,
+                    amax_out: torch.Tensor | None = None, overflow: int = SATURATE) -> None:
+    """D[M,N] (uint8 codes of format fd) = encode((A . B) * scale_inv_a * scale_inv_b * scale_d); amax_out
+    receives the amax of the result before the output scale and conversion.  Layout rules as fp8_gemm."""
+    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or D.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
+        raise TypeError("A, B and D must be 2-D uint8 tensors")
+    for t, name in ((A, "A"), (B, "B"), (D, "D")):
+        if not t.is_cuda or t.stride(1) != 1:
+            raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
+    M, K = (A.shape[0], A.shape[1]) if ma == MAJOR_K else (A.shape[1], A.shape[0])
+    Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
+    if K != Kb or tuple(D.shape) != (M, N):
+        raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
+    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), BF16)
+    _check(load().fp8_gemm_fp8out(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(), fd, overflow,
+                                  _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
+                                  _scalar(scale_d, "scale_d"), None if amax_out is None else _scalar(amax_out, "amax_out"),
+                                  _stream()), "fp8_gemm_fp8out")
 
 
 def fp8_async_status() -> tuple[int, int]:

@@ -247,7 +247,47 @@ struct Params {
     uint32_t* amax_bits;            // may be null
     uint32_t idesc;                 // M field set for the CTA group the kernel was built for
     int tiles_m, tiles_n;           // tiles of (128*CG) x 256
+    int a_mn, b_mn;                 // operand stored with its M (resp. N) index contiguous
+    const float* scale_d;           // FP8 output only: scale applied before the conversion
+    int nosat;                      // FP8 output only: non-saturating conversion
 };
+
+// what the epilogue writes
+constexpr int OUT_F32 = 0, OUT_BF16 = 1, OUT_E4M3 = 2, OUT_E5M2 = 3;
+
+// 32 accumulator values (already multiplied by alpha) -> 32 FP8 codes of y = v * scale_d, packed in 8 words.
+// Same rules as the cast kernels: hardware convert unless a special value (or, non-saturating, an overflow)
+// is present; a NaN code takes the sign of v.
+template <int FMT>
+__device__ __forceinline__ void encode32(const float (&v)[32], float scale_d, bool nosat, uint32_t (&w)[8]) {
+    float y[32];
+    float poison = 0.0f, top = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        y[i] = v[i] * scale_d;
+        poison = fmaf(y[i], 0.0f, poison);
+        top = fmaxf(top, fabsf(y[i]));
+    }
+    const bool over = Fmt<FMT>::nosat_limit_inclusive ? top >= Fmt<FMT>::nosat_limit : top > Fmt<FMT>::nosat_limit;
+    if (poison == poison && !(nosat && over)) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) w[q] = cvt_quad<FMT>(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+    } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t word = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const float yy = y[4 * q + b];
+                uint32_t code;
+                if (yy != yy) code = ((__float_as_uint(v[4 * q + b]) >> 24) & 0x80u) | 0x7Fu;
+                else code = nosat ? encode_scalar<FMT, true>(yy) : encode_scalar<FMT, false>(yy);
+                word |= code << (8 * b);
+            }
+            w[q] = word;
+        }
+    }
+}
 
 struct alignas(8) Barriers {
     uint64_t full[MAX_STAGES];
@@ -271,9 +311,10 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
     tn = r / rows;
 }
 
-// CG: CTAs per tile (1 or 2).  A_MN / B_MN: operand stored with its M (resp. N) index contiguous.
-// OUT_BF16: D is bf16, else fp32.
-template <int CG, bool A_MN, bool B_MN, bool OUT_BF16>
+// CG: CTAs per tile (1 or 2).  OUT: what the epilogue writes (fp32, bf16, E4M3 or E5M2 codes).
+// Operand layouts (K-major or MN-major) are run-time properties: they only change TMA coordinates and
+// shared-memory descriptor constants.
+template <int CG, int OUT>
 __global__ void __launch_bounds__(THREADS, 1)
 k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
            const __grid_constant__ CUtensorMap map_d, const Params p) {
@@ -292,6 +333,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
     const int worker = blockIdx.x / CG, num_workers = gridDim.x / CG;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int k_blocks = (int)((p.K + BK - 1) / BK);
+    const bool A_MN = p.a_mn != 0, B_MN = p.b_mn != 0;
     constexpr int FG = G::FG;
     const int k_pad = (k_blocks + FG - 1) / FG * FG;               // K-blocks are consumed FG at a time
 
@@ -374,6 +416,8 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         uint32_t stage = 0, phase = 0;
         bool ok = cta_rank == 0;
         int it = 0;
+        const uint32_t a_kstep = A_MN ? UMMA_K * 128 : UMMA_K, a_lbo = A_MN ? BK * 128 : 16;
+        const uint32_t b_kstep = B_MN ? UMMA_K * 128 : UMMA_K, b_lbo = B_MN ? BK * 128 : 16;
         PROF_DECL
         for (int t = worker; t < num_tiles && ok; t += num_workers, ++it) {
             const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
@@ -401,10 +445,8 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                             for (int k = 0; k < BK / UMMA_K; ++k) {
                                 // K-major: 8-row groups 1024 B apart, +32 B per K step inside the swizzled row.
                                 // MN-major: 8-k groups 1024 B apart, 128-wide MN blocks BK*128 B apart, +32 k-rows per step.
-                                const uint64_t da = A_MN ? smem_desc(sa + k * UMMA_K * 128, BK * 128, 1024)
-                                                         : smem_desc(sa + k * UMMA_K, 16, 1024);
-                                const uint64_t db = B_MN ? smem_desc(sb + k * UMMA_K * 128, BK * 128, 1024)
-                                                         : smem_desc(sb + k * UMMA_K, 16, 1024);
+                                const uint64_t da = smem_desc(sa + k * a_kstep, a_lbo, 1024);
+                                const uint64_t db = smem_desc(sb + k * b_kstep, b_lbo, 1024);
                                 if (CG == 2) tc_mma_f8_pair(tmem_d, da, db, p.idesc, (kb | h | k) != 0 ? 1u : 0u);
                                 else         tc_mma_f8(tmem_d, da, db, p.idesc, (kb | h | k) != 0 ? 1u : 0u);
                             }
@@ -430,6 +472,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         // ------------------------------------------------------------ epilogue (each CTA drains its own 128 rows)
         const int q = warp & 3;                                   // TMEM lane quarter this warp may read
         const float alpha = __ldg(p.sa_inv) * __ldg(p.sb_inv);
+        const float scale_d = (OUT == OUT_E4M3 || OUT == OUT_E5M2) ? __ldg(p.scale_d) : 1.0f;
         uint32_t running = 0;                                     // max of stored magnitude bits (bf16: 16-bit patterns)
         const uint32_t epi_base = ring + SMEM_TILES + (uint32_t)(warp - 2) * 2u * EPI_BUF_BYTES;
         uint32_t buf = 0;
@@ -450,61 +493,82 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             const bool row_ok = (int64_t)row0 + lane < p.M;
             const int64_t col0 = (int64_t)tn * BN;
             const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
-            constexpr int CHUNK = OUT_BF16 ? 64 : 32;             // columns per staged box: 128 bytes per row
-            constexpr int ESZ = OUT_BF16 ? 2 : 4;
+            constexpr int ESZ = OUT == OUT_F32 ? 4 : OUT == OUT_BF16 ? 2 : 1;
+            constexpr int CHUNK = 128 / ESZ;                      // columns per staged box: 128 bytes per row
+            constexpr int SUBS = CHUNK / 32;                      // 32-column TMEM loads per box
+            constexpr int WORDS = 32 * ESZ / 4;                   // 32-bit words one load contributes to the row
 #pragma unroll 1
             for (int c = 0; c < BN / CHUNK; ++c) {
-                uint32_t w[32];                                   // the 128 bytes this thread contributes to its row
-                if (OUT_BF16) {
-                    uint32_t r0[32], r1[32];
-                    tc_ld32(taddr + c * 64, r0);
-                    tc_ld32(taddr + c * 64 + 32, r1);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        w[i] = pack_bf16(__uint_as_float(r0[2 * i]) * alpha, __uint_as_float(r0[2 * i + 1]) * alpha);
-                        w[16 + i] = pack_bf16(__uint_as_float(r1[2 * i]) * alpha, __uint_as_float(r1[2 * i + 1]) * alpha);
-                    }
-                } else {
-                    tc_ld32(taddr + c * 32, w);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
-                }
                 const int64_t col = col0 + (int64_t)c * CHUNK;
-                if (row_ok && col < p.N) {                        // amax over in-bounds elements only
-                    if (col + CHUNK <= p.N) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            running = OUT_BF16 ? __vmaxu2(running, w[i] & 0x7FFF7FFFu) : max(running, w[i] & 0x7FFFFFFFu);
-                    } else {
-                        for (int i = 0; i < CHUNK && col + i < p.N; ++i) {
-                            const uint32_t h = OUT_BF16 ? (((i & 1) ? (w[i >> 1] >> 16) : w[i >> 1]) & 0x7FFFu) : (w[i] & 0x7FFFFFFFu);
-                            running = OUT_BF16 ? __vmaxu2(running, h) : max(running, h);
-                        }
-                    }
-                }
                 // A box that crosses the right edge is clipped by the TMA unit in 16-byte units: when the row
                 // length in bytes is not a multiple of 16 that last box is written with plain stores instead.
-                const bool clipped_mid_16 = col + CHUNK > p.N && ((p.N * ESZ) & 15) != 0;
-                if (clipped_mid_16) {
-                    if (row_ok) {
-                        for (int i = 0; i < CHUNK && col + i < p.N; ++i) {
-                            if (OUT_BF16) reinterpret_cast<uint16_t*>(p.D)[((int64_t)row0 + lane) * p.ldd + col + i] =
-                                              (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : w[i >> 1]);
-                            else          reinterpret_cast<uint32_t*>(p.D)[((int64_t)row0 + lane) * p.ldd + col + i] = w[i];
-                        }
-                    }
-                    continue;
-                }
-                // stage the 32 x 128 B box with the 128-byte swizzle the tensor map expects, then store it
-                if (lane == 0) bulk_wait_read<1>();               // the box stored two chunks ago has left this buffer
-                __syncwarp();
+                const bool direct = col + CHUNK > p.N && ((p.N * ESZ) & 15) != 0;
                 const uint32_t sbuf = epi_base + buf * EPI_BUF_BYTES;
                 const uint32_t srow = sbuf + lane * 128;
+                if (!direct) {
+                    if (lane == 0) bulk_wait_read<1>();           // the box stored two chunks ago has left this buffer
+                    __syncwarp();
+                }
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    st_shared_v4(srow + ((j ^ (lane & 7)) << 4), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                for (int sub = 0; sub < SUBS; ++sub) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + c * CHUNK + sub * 32, r);
+                    tc_wait_ld();
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * alpha;
+                    uint32_t w[WORDS];                            // this thread's bytes of its row for these 32 columns
+                    if (OUT == OUT_F32) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(v[i]);
+                    } else if (OUT == OUT_BF16) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) w[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+                    } else {
+                        uint32_t codes[8];
+                        if (OUT == OUT_E4M3) encode32<kE4M3>(v, scale_d, p.nosat != 0, codes);
+                        else                 encode32<kE5M2>(v, scale_d, p.nosat != 0, codes);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) w[i] = codes[i];
+                    }
+                    // amax over in-bounds elements: of the stored values (fp32, bf16), of v before the output
+                    // scale and conversion (FP8 output)
+                    const int64_t scol = col + sub * 32;
+                    if (row_ok && scol < p.N) {
+                        if (scol + 32 <= p.N) {
+                            if (OUT == OUT_BF16) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) running = __vmaxu2(running, w[i] & 0x7FFF7FFFu);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) running = max(running, __float_as_uint(v[i]) & 0x7FFFFFFFu);
+                            }
+                        } else {
+                            for (int i = 0; i < 32 && scol + i < p.N; ++i) {
+                                if (OUT == OUT_BF16) running = __vmaxu2(running, ((i & 1) ? (w[i >> 1] >> 16) : w[i >> 1]) & 0x7FFFu);
+                                else                 running = max(running, __float_as_uint(v[i]) & 0x7FFFFFFFu);
+                            }
+                        }
+                    }
+                    if (direct) {
+                        if (row_ok) {
+                            uint8_t* drow = reinterpret_cast<uint8_t*>(p.D) + (((int64_t)row0 + lane) * p.ldd + scol) * ESZ;
+                            for (int i = 0; i < 32 && scol + i < p.N; ++i) {
+                                if (OUT == OUT_F32)       reinterpret_cast<uint32_t*>(drow)[i] = w[i];
+                                else if (OUT == OUT_BF16) reinterpret_cast<uint16_t*>(drow)[i] = (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : w[i >> 1]);
+                                else                      drow[i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
+                            }
+                        }
+                    } else {
+                        // the 32 x 128 B box is staged with the 128-byte swizzle the tensor map expects
+#pragma unroll
+                        for (int j = 0; j < WORDS / 4; ++j) {
+                            const int pos = sub * (WORDS / 4) + j;            // 16-byte position inside the 128-byte row
+                            st_shared_v4(srow + ((pos ^ (lane & 7)) << 4), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                        }
+                    }
+                }
+                if (direct) continue;
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
@@ -523,7 +587,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         if (lane == 0) bulk_wait_all();                           // every store has reached global memory before exit
         if (warp == 2) { PROF_STORE(6, 7, -1) }
         if (p.amax_bits) {
-            uint32_t bits = OUT_BF16 ? (max(running & 0xFFFFu, running >> 16) << 16) : running;
+            uint32_t bits = OUT == OUT_BF16 ? (max(running & 0xFFFFu, running >> 16) << 16) : running;
             bits = warp_max_u32(canonical_nan_bits(bits));
             if (lane == 0 && bits != 0u) atomicMax(p.amax_bits, bits);
         }
@@ -536,17 +600,6 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         tc_fence_after();
         if (CG == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
         else         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-    }
-}
-
-// K == 0: D = 0.
-template <bool OUT_BF16>
-__global__ void k_zero_d(void* D, int64_t M, int64_t N, int64_t ldd) {
-    const int64_t total = M * N;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = i / N, c = i - r * N;
-        if (OUT_BF16) reinterpret_cast<uint16_t*>(D)[r * ldd + c] = 0;
-        else          reinterpret_cast<float*>(D)[r * ldd + c] = 0.0f;
     }
 }
 
@@ -584,9 +637,9 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
 }
 
 // CTA-pair kernels launch as clusters of 2; the grid is one CTA per SM that can be paired.
-template <int CG, bool A_MN, bool B_MN, bool OUT_BF16>
+template <int CG, int OUT>
 static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const Params& p, int64_t num_tiles, cudaStream_t st) {
-    auto k = k_gemm_fp8<CG, A_MN, B_MN, OUT_BF16>;
+    auto k = k_gemm_fp8<CG, OUT>;
     // per device and cheap, so set on every launch rather than cached
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return FP8_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -615,34 +668,23 @@ static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
 }
 
 template <int CG>
-static fp8_status dispatch(bool a_mn, bool b_mn, bool bf, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
+static fp8_status dispatch(int out_kind, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
                            const Params& p, int64_t num_tiles, cudaStream_t st) {
-    if (!a_mn && !b_mn) return bf ? launch<CG, false, false, true>(ma, mb, md, p, num_tiles, st) : launch<CG, false, false, false>(ma, mb, md, p, num_tiles, st);
-    if (!a_mn && b_mn)  return bf ? launch<CG, false, true, true>(ma, mb, md, p, num_tiles, st)  : launch<CG, false, true, false>(ma, mb, md, p, num_tiles, st);
-    if (a_mn && !b_mn)  return bf ? launch<CG, true, false, true>(ma, mb, md, p, num_tiles, st)  : launch<CG, true, false, false>(ma, mb, md, p, num_tiles, st);
-    return bf ? launch<CG, true, true, true>(ma, mb, md, p, num_tiles, st) : launch<CG, true, true, false>(ma, mb, md, p, num_tiles, st);
+    switch (out_kind) {
+        case OUT_F32:  return launch<CG, OUT_F32>(ma, mb, md, p, num_tiles, st);
+        case OUT_BF16: return launch<CG, OUT_BF16>(ma, mb, md, p, num_tiles, st);
+        case OUT_E4M3: return launch<CG, OUT_E4M3>(ma, mb, md, p, num_tiles, st);
+        default:       return launch<CG, OUT_E5M2>(ma, mb, md, p, num_tiles, st);
+    }
 }
 
-}  // namespace gemm
-}  // namespace fp8b200
-
-using namespace fp8b200;
-
-extern "C" {
-
-fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,
-                    const float* scale_inv_a_dev, const float* scale_inv_b_dev, float* amax_d_dev, void* stream) {
-    using namespace fp8b200::gemm;
-    if (!d || !scale_inv_a_dev || !scale_inv_b_dev) return FP8_ERR_NULL;
-    if ((d->fa != FP8_E4M3 && d->fa != FP8_E5M2) || (d->fb != FP8_E4M3 && d->fb != FP8_E5M2) ||
-        (d->ma != FP8_MAJOR_K && d->ma != FP8_MAJOR_MN) || (d->mb != FP8_MAJOR_K && d->mb != FP8_MAJOR_MN) ||
-        (d->out != FP8_F32 && d->out != FP8_BF16))
-        return FP8_ERR_ENUM;
+// Shared body of fp8_gemm and fp8_gemm_fp8out.
+static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D, int out_kind, int nosat,
+                            const float* sa_inv, const float* sb_inv, const float* scale_d, float* amax_d_dev, cudaStream_t st) {
     const int64_t M = d->M, N = d->N, K = d->K;
     if (M < 0 || N < 0 || K < 0) return FP8_ERR_SHAPE;
-    cudaStream_t st = (cudaStream_t)stream;
     const bool a_mn = d->ma == FP8_MAJOR_MN, b_mn = d->mb == FP8_MAJOR_MN;
-    const int64_t esz = d->out == FP8_BF16 ? 2 : 4;
+    const int64_t esz = out_kind == OUT_F32 ? 4 : out_kind == OUT_BF16 ? 2 : 1;
     // CTA pairs (256-row tiles) unless the whole problem has at most 128 rows
     const int cg = M > BM ? 2 : 1;
     const int64_t tile_m = (int64_t)BM * cg;
@@ -668,12 +710,10 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
         count_launches(1);
     }
     if (M == 0 || N == 0) return FP8_OK;
-    if (K == 0) {
-        const int grid = sm_count() * 4;
-        if (d->out == FP8_BF16) k_zero_d<true><<<grid, 256, 0, st>>>(D, M, N, d->ldd);
-        else                    k_zero_d<false><<<grid, 256, 0, st>>>(D, M, N, d->ldd);
+    if (K == 0) {                                                 // empty sum: zeros in every output type
+        if (cudaMemset2DAsync(D, (size_t)(d->ldd * esz), 0, (size_t)(N * esz), (size_t)M, st) != cudaSuccess) return FP8_ERR_CUDA;
         count_launches(1);
-        return launch_status();
+        return FP8_OK;
     }
 
     CUtensorMap map_a, map_b;
@@ -689,15 +729,47 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
 
     Params p;
     p.M = M; p.N = N; p.K = K; p.ldd = d->ldd; p.D = D;
-    p.sa_inv = scale_inv_a_dev; p.sb_inv = scale_inv_b_dev;
+    p.sa_inv = sa_inv; p.sb_inv = sb_inv;
     p.amax_bits = reinterpret_cast<uint32_t*>(amax_d_dev);
     p.tiles_m = (int)tiles_m; p.tiles_n = (int)tiles_n;
+    p.a_mn = a_mn ? 1 : 0; p.b_mn = b_mn ? 1 : 0;
+    p.scale_d = scale_d; p.nosat = nosat;
     // instruction descriptor: fp32 accumulate, operand formats and majors, N/8, M/16 (M = 256 for a CTA pair)
     p.idesc = (1u << 4) | ((uint32_t)d->fa << 7) | ((uint32_t)d->fb << 10) | ((a_mn ? 1u : 0u) << 15) |
               ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
-    const bool bf = d->out == FP8_BF16;
-    return cg == 2 ? dispatch<2>(a_mn, b_mn, bf, map_a, map_b, map_d, p, tiles_m * tiles_n, st)
-                   : dispatch<1>(a_mn, b_mn, bf, map_a, map_b, map_d, p, tiles_m * tiles_n, st);
+    return cg == 2 ? dispatch<2>(out_kind, map_a, map_b, map_d, p, tiles_m * tiles_n, st)
+                   : dispatch<1>(out_kind, map_a, map_b, map_d, p, tiles_m * tiles_n, st);
+}
+
+}  // namespace gemm
+}  // namespace fp8b200
+
+using namespace fp8b200;
+
+extern "C" {
+
+static bool desc_enums_ok(const fp8_gemm_desc* d) {
+    return (d->fa == FP8_E4M3 || d->fa == FP8_E5M2) && (d->fb == FP8_E4M3 || d->fb == FP8_E5M2) &&
+           (d->ma == FP8_MAJOR_K || d->ma == FP8_MAJOR_MN) && (d->mb == FP8_MAJOR_K || d->mb == FP8_MAJOR_MN);
+}
+
+fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,
+                    const float* scale_inv_a_dev, const float* scale_inv_b_dev, float* amax_d_dev, void* stream) {
+    using namespace fp8b200::gemm;
+    if (!d || !scale_inv_a_dev || !scale_inv_b_dev) return FP8_ERR_NULL;
+    if (!desc_enums_ok(d) || (d->out != FP8_F32 && d->out != FP8_BF16)) return FP8_ERR_ENUM;
+    return gemm_impl(d, A, B, D, d->out == FP8_BF16 ? OUT_BF16 : OUT_F32, 0, scale_inv_a_dev, scale_inv_b_dev, nullptr,
+                     amax_d_dev, (cudaStream_t)stream);
+}
+
+fp8_status fp8_gemm_fp8out(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, uint8_t* D, fp8_format fd, fp8_overflow od,
+                           const float* scale_inv_a_dev, const float* scale_inv_b_dev, const float* scale_d_dev,
+                           float* amax_d_dev, void* stream) {
+    using namespace fp8b200::gemm;
+    if (!d || !scale_inv_a_dev || !scale_inv_b_dev || !scale_d_dev) return FP8_ERR_NULL;
+    if (!desc_enums_ok(d) || (fd != FP8_E4M3 && fd != FP8_E5M2) || (od != FP8_SATURATE && od != FP8_NOSAT)) return FP8_ERR_ENUM;
+    return gemm_impl(d, A, B, D, fd == FP8_E4M3 ? OUT_E4M3 : OUT_E5M2, od == FP8_NOSAT ? 1 : 0, scale_inv_a_dev, scale_inv_b_dev,
+                     scale_d_dev, amax_d_dev, (cudaStream_t)stream);
 }
 
 #ifdef FP8_GEMM_PROFILE

@@ -67,3 +67,27 @@ def check_gemm_bf16(gpu_bits: np.ndarray, ref: np.ndarray, sabs: np.ndarray, rou
         ok = np.where(special, sp_ok, ok)
         literal = np.where(special, sp_ok, literal)
     return ok, literal
+
+
+def fp8_order(codes: np.ndarray) -> np.ndarray:
+    """FP8 codes -> integers ordered like the values (sign-magnitude; both zeros map to 0)"""
+    c = codes.astype(np.int64)
+    return np.where(c & 0x80, -(c & 0x7F), c & 0x7F)
+
+
+def check_gemm_fp8out(gpu_codes: np.ndarray, ref: np.ndarray, sabs: np.ndarray, scale_d: float, encode, rel: float = 1e-5):
+    """FP8-output criterion: the stored code lies within one code of encode(v * scale_d) for some v in
+    [ref - rel*sabs, ref + rel*sabs] (encode is monotonic, so that set is a code interval).
+    `encode(float32 array) -> codes` is the oracle's conversion.  NaN reference -> NaN code."""
+    special = ~np.isfinite(ref)
+    tol = rel * sabs
+    sd = np.float64(scale_d)
+    with np.errstate(over="ignore", invalid="ignore"):
+        lo = fp8_order(encode(np.where(special, 0.0, (ref - tol) * sd).astype(np.float32)))
+        hi = fp8_order(encode(np.where(special, 0.0, (ref + tol) * sd).astype(np.float32)))
+    g = fp8_order(gpu_codes)
+    ok = (g >= lo - 1) & (g <= hi + 1)
+    if special.any():
+        want = encode(np.where(special, ref * sd, 0.0).astype(np.float32))
+        ok = np.where(special, gpu_codes == want, ok)
+    return ok

@@ -8,7 +8,7 @@ import torch
 
 import oracle
 from paper_2209_05433_b200 import api, synth
-from tests._util import THREADS, check_gemm_bf16, check_gemm_f32, to_np_bits
+from tests._util import THREADS, check_gemm_bf16, check_gemm_f32, check_gemm_fp8out, to_np_bits
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -218,3 +218,73 @@ def test_special_codes_and_degenerate_shapes():
     Bz = torch.empty((64, 32), dtype=torch.uint8, device=DEV)
     api.fp8_gemm(Az, E4, api.MAJOR_K, Bz, E4, api.MAJOR_K, Dz, _scalar(1.0), _scalar(1.0), amax)
     assert amax.item() == 0.0
+
+
+# ------------------------------------------------ FP8-output epilogue --
+
+@pytest.mark.parametrize("role", list(ROLES))
+@pytest.mark.parametrize("fd", [E4, E5])
+@pytest.mark.parametrize("shape", [(384, 768, 640), (129, 257, 129), (100, 40, 48), (300, 520, 200)])
+def test_fp8_output_epilogue(role, fd, shape):
+    """results converted to FP8 before they are written; amax reported before the output scale"""
+    fa, fb = ROLES[role]
+    M, N, K = shape
+    rng = np.random.default_rng(2000 + list(ROLES).index(role) * 8 + fd * 4 + M)
+    ma, mb = (api.MAJOR_K, api.MAJOR_MN) if role == "fprop" else (api.MAJOR_K, api.MAJOR_K) if role == "dgrad" else (api.MAJOR_MN, api.MAJOR_MN)
+    A_np = _codes(rng, fa, (M, K) if ma == api.MAJOR_K else (K, M))
+    B_np = _codes(rng, fb, (N, K) if mb == api.MAJOR_K else (K, N))
+    A_buf, B_buf = _pad_cols(A_np), _pad_cols(B_np)
+    A = torch.from_numpy(A_buf).to(DEV)[:, : A_np.shape[1]]
+    B = torch.from_numpy(B_buf).to(DEV)[:, : B_np.shape[1]]
+    ldd = (N + 15) // 16 * 16
+    sa_inv, sb_inv = 0.013, 0.5
+    a_str = (A_buf.shape[1], 1) if ma == api.MAJOR_K else (1, A_buf.shape[1])
+    b_str = (1, B_buf.shape[1]) if mb == api.MAJOR_K else (B_buf.shape[1], 1)
+    ref, sabs = oracle.gemm_rows(A_buf, fa, a_str, B_buf, fb, b_str, N, K, 0, M, sa_inv, sb_inv, threads=THREADS)
+    want_amax = np.abs(ref).max()
+    # a scale chosen as the method would: from (an estimate of) the output's own maximum; and one that overflows
+    for scale_d, overflow in ((float(oracle.scale_from_amax(np.float32(want_amax), fd)[0]), api.SATURATE),
+                              (float(oracle.scale_from_amax(np.float32(want_amax), fd)[0]) * 8.0, api.SATURATE),
+                              (float(oracle.scale_from_amax(np.float32(want_amax), fd)[0]) * 8.0, api.NOSAT)):
+        D_full = torch.full((M + 1, ldd), 0xA5, dtype=torch.uint8, device=DEV)
+        D = D_full[:M, :N]
+        amax = _scalar(-1.0)
+        api.fp8_gemm_fp8out(A, fa, ma, B, fb, mb, D, fd, _scalar(sa_inv), _scalar(sb_inv), _scalar(scale_d), amax, overflow)
+        torch.cuda.synchronize()
+        assert api.fp8_async_status()[0] == 0
+        assert bool((D_full[M:, :] == 0xA5).all()) and bool((D_full[:M, N:] == 0xA5).all()), "wrote outside D"
+        enc = lambda y: oracle.quantize(y.reshape(-1), 1.0, fd, overflow, threads=THREADS).reshape(y.shape)
+        ok = check_gemm_fp8out(D.cpu().numpy(), ref, sabs, scale_d, enc)
+        assert ok.all(), "%d of %d codes out of tolerance at %s" % ((~ok).sum(), ok.size, np.argwhere(~ok)[:4].tolist())
+        # amax of the unscaled, unconverted result: within the accumulation tolerance of the oracle's
+        got_amax = float(amax.item())
+        lo = np.max(np.abs(ref) - 1e-5 * sabs) * (1 - 2.0 ** -22)
+        hi = np.max(np.abs(ref) + 1e-5 * sabs) * (1 + 2.0 ** -22)
+        assert lo <= got_amax <= hi, (got_amax, lo, hi)
+
+
+def test_fp8_output_special_values_and_k0():
+    rng = np.random.default_rng(31)
+    M, N, K = 256, 256, 128
+    A_np = _codes(rng, E5, (M, K))
+    B_np = _codes(rng, E4, (N, K))
+    A_np[3, 7] = 0x7C          # +Inf  -> row 3 is +-Inf or NaN
+    B_np[40, 100] = 0x7F       # NaN   -> column 40 is NaN
+    A = torch.from_numpy(A_np).to(DEV)
+    B = torch.from_numpy(B_np).to(DEV)
+    ref, sabs = oracle.gemm_rows(A_np, E5, (K, 1), B_np, E4, (1, K), N, K, 0, M, 1.0, 1.0, threads=THREADS)
+    for fd in (E4, E5):
+        D = torch.empty(M, N, dtype=torch.uint8, device=DEV)
+        api.fp8_gemm_fp8out(A, E5, api.MAJOR_K, B, E4, api.MAJOR_K, D, fd, _scalar(1.0), _scalar(1.0), _scalar(0.01))
+        enc = lambda y: oracle.quantize(y.reshape(-1), 1.0, fd, threads=THREADS).reshape(y.shape)
+        ok = check_gemm_fp8out(D.cpu().numpy(), ref, sabs, 0.01, enc)
+        assert ok.all(), np.argwhere(~ok)[:4].tolist()
+        got = D.cpu().numpy()
+        assert ((got[:, 40] & 0x7F) == 0x7F).all()                      # NaN codes
+        inf_row = got[3, np.isinf(ref[3])]
+        assert ((inf_row & 0x7F) == (0x7F if fd == E4 else 0x7C)).all()  # Inf -> NaN (E4M3) / Inf (E5M2), never the maximum
+    D = torch.full((64, 64), 0x11, dtype=torch.uint8, device=DEV)
+    amax = _scalar(3.0)
+    A0 = torch.empty((64, 0), dtype=torch.uint8, device=DEV)
+    api.fp8_gemm_fp8out(A0, E4, api.MAJOR_K, A0, E4, api.MAJOR_K, D, E4, _scalar(1.0), _scalar(1.0), _scalar(1.0), amax)
+    assert bool((D == 0).all()) and amax.item() == 0.0
