@@ -83,6 +83,18 @@ def _load():
     lib.fp8o_gemm_rows.restype = None
     lib.fp8o_gemm_rows.argtypes = gemm_common + [c.c_int64, c.c_int64, c.c_int64, c.c_int64,
                                                  c.c_float, c.c_float, f64p, f64p]
+    u32p = c.POINTER(c.c_uint32)
+    lib.fp8o_amax_channels_f32.restype = None
+    lib.fp8o_amax_channels_f32.argtypes = [f32p, c.c_int64, c.c_int64, c.c_int64, c.c_int, u32p]
+    lib.fp8o_amax_channels_bf16.restype = None
+    lib.fp8o_amax_channels_bf16.argtypes = [u16p, c.c_int64, c.c_int64, c.c_int64, c.c_int, u32p]
+    lib.fp8o_quantize_channels_f32.restype = None
+    lib.fp8o_quantize_channels_f32.argtypes = [f32p, c.c_int64, c.c_int64, c.c_int64, c.c_int, f32p, c.c_int, c.c_int, u8p, c.c_int64]
+    lib.fp8o_quantize_channels_bf16.restype = None
+    lib.fp8o_quantize_channels_bf16.argtypes = [u16p, c.c_int64, c.c_int64, c.c_int64, c.c_int, f32p, c.c_int, c.c_int, u8p, c.c_int64]
+    lib.fp8o_gemm_rows_colscale.restype = None
+    lib.fp8o_gemm_rows_colscale.argtypes = gemm_common + [c.c_int64, c.c_int64, c.c_int64, c.c_int64,
+                                                          c.c_float, f32p, f64p, f64p]
     lib.fp8o_gemm_samples.restype = None
     lib.fp8o_gemm_samples.argtypes = gemm_common + [c.c_int64, i64p, i64p, c.c_int64,
                                                     c.c_float, c.c_float, f64p, f64p]
@@ -225,6 +237,67 @@ def amax_bits(x: np.ndarray, threads: int = 1) -> int:
 
 def amax(x: np.ndarray, threads: int = 1) -> np.float32:
     return np.array([amax_bits(x, threads)], dtype=np.uint32).view(np.float32)[0]
+
+
+# ------------------------------------------------------- per-channel scales --
+
+def amax_channels(x: np.ndarray, axis: int) -> np.ndarray:
+    """float32 amax per channel of a 2-D array: axis 0 = one per column, axis 1 = one per row."""
+    lib = _load()
+    x = np.ascontiguousarray(x)
+    rows, cols = x.shape
+    out = np.empty(cols if axis == 0 else rows, dtype=np.uint32)
+    if _wide_kind(x.reshape(-1)) == "f32":
+        lib.fp8o_amax_channels_f32(_ptr(x, ctypes.c_float), rows, cols, cols, axis, _ptr(out, ctypes.c_uint32))
+    else:
+        lib.fp8o_amax_channels_bf16(_ptr(x, ctypes.c_uint16), rows, cols, cols, axis, _ptr(out, ctypes.c_uint32))
+    return out.view(np.float32)
+
+
+def scales_from_amax(amax_vec: np.ndarray, fmt: int, pow2: bool = False):
+    s = np.empty(amax_vec.size, dtype=np.float32)
+    si = np.empty(amax_vec.size, dtype=np.float32)
+    for i, a in enumerate(np.asarray(amax_vec, dtype=np.float32).reshape(-1)):
+        s[i], si[i] = scale_pow2_from_amax(a, fmt) if pow2 else scale_from_amax(a, fmt)
+    return s, si
+
+
+def quantize_channels(x: np.ndarray, scale_vec: np.ndarray, axis: int, fmt: int, overflow: int = SATURATE) -> np.ndarray:
+    lib = _load()
+    x = np.ascontiguousarray(x)
+    rows, cols = x.shape
+    sv = np.ascontiguousarray(scale_vec, dtype=np.float32)
+    assert sv.size == (cols if axis == 0 else rows)
+    out = np.empty((rows, cols), dtype=np.uint8)
+    if _wide_kind(x.reshape(-1)) == "f32":
+        lib.fp8o_quantize_channels_f32(_ptr(x, ctypes.c_float), rows, cols, cols, axis, _ptr(sv, ctypes.c_float), fmt, overflow,
+                                       _ptr(out, ctypes.c_uint8), cols)
+    else:
+        lib.fp8o_quantize_channels_bf16(_ptr(x, ctypes.c_uint16), rows, cols, cols, axis, _ptr(sv, ctypes.c_float), fmt, overflow,
+                                        _ptr(out, ctypes.c_uint8), cols)
+    return out
+
+
+def gemm_rows_colscale(A, fmt_a, a_strides, B, fmt_b, b_strides, N, K, i0, i1, sa_inv, sb_inv_vec, threads: int = 1):
+    """gemm_rows with one inverse scale per column of B (per output channel)."""
+    lib = _load()
+    A = np.ascontiguousarray(A, dtype=np.uint8).reshape(-1)
+    B = np.ascontiguousarray(B, dtype=np.uint8).reshape(-1)
+    sv = np.ascontiguousarray(sb_inv_vec, dtype=np.float32)
+    assert sv.size == N
+    rows = i1 - i0
+    ref = np.empty((rows, N), dtype=np.float64)
+    sab = np.empty((rows, N), dtype=np.float64)
+    sa = ctypes.c_float(np.float32(sa_inv))
+    jobs = []
+    for lo, hi in _chunks(rows, threads):
+        jobs.append(lambda lo=lo, hi=hi: lib.fp8o_gemm_rows_colscale(
+            _ptr(A, ctypes.c_uint8), fmt_a, a_strides[0], a_strides[1],
+            _ptr(B, ctypes.c_uint8), fmt_b, b_strides[0], b_strides[1],
+            N, K, i0 + lo, i0 + hi, sa, _ptr(sv, ctypes.c_float),
+            _ptr(ref[lo:hi], ctypes.c_double), _ptr(sab[lo:hi], ctypes.c_double)))
+    _run(jobs, threads)
+    return ref, sab
 
 
 # --------------------------------------------------------------------- GEMM --

@@ -283,6 +283,61 @@ void fp8o_scale_pow2_from_amax(float amax, int fmt, float* scale, float* scale_i
     *scale_inv = (float)(1.0 / (double)s);
 }
 
+/* ------------------------------------------------------ per-channel scales */
+
+/* Section 4.2: "per-channel scaling factors for weights, per-tensor scaling
+ * factors for activations".  x is rows x cols, row-major with pitch ld (in
+ * elements).  axis 0: one channel per column (the maximum runs over rows);
+ * axis 1: one channel per row.  Same definition as the per-tensor amax. */
+void fp8o_amax_channels_f32(const float* x, int64_t rows, int64_t cols, int64_t ld, int axis, uint32_t* amax_bits)
+{
+    int64_t channels = axis == 0 ? cols : rows, len = axis == 0 ? rows : cols;
+    for (int64_t c = 0; c < channels; ++c) {
+        int saw_nan = 0;
+        float best = 0.0f;
+        for (int64_t i = 0; i < len; ++i) {
+            float v = axis == 0 ? x[i * ld + c] : x[c * ld + i];
+            if (isnan(v)) { saw_nan = 1; continue; }
+            float a = fabsf(v);
+            if (a > best) best = a;
+        }
+        amax_bits[c] = saw_nan ? 0x7FC00000u : f32_bits(best);
+    }
+}
+
+void fp8o_amax_channels_bf16(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld, int axis, uint32_t* amax_bits)
+{
+    int64_t channels = axis == 0 ? cols : rows, len = axis == 0 ? rows : cols;
+    for (int64_t c = 0; c < channels; ++c) {
+        int saw_nan = 0;
+        float best = 0.0f;
+        for (int64_t i = 0; i < len; ++i) {
+            float v = bf16_to_f32(axis == 0 ? x[i * ld + c] : x[c * ld + i]);
+            if (isnan(v)) { saw_nan = 1; continue; }
+            float a = fabsf(v);
+            if (a > best) best = a;
+        }
+        amax_bits[c] = saw_nan ? 0x7FC00000u : f32_bits(best);
+    }
+}
+
+/* out[r*ld_out + c] = encode( x[r*ld + c] * scale[channel of (r,c)] ) */
+void fp8o_quantize_channels_f32(const float* x, int64_t rows, int64_t cols, int64_t ld, int axis, const float* scale,
+                                int fmt, int overflow, uint8_t* out, int64_t ld_out)
+{
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < cols; ++c)
+            out[r * ld_out + c] = quantize_one(x[r * ld + c], scale[axis == 0 ? c : r], fmt, overflow);
+}
+
+void fp8o_quantize_channels_bf16(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld, int axis, const float* scale,
+                                 int fmt, int overflow, uint8_t* out, int64_t ld_out)
+{
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < cols; ++c)
+            out[r * ld_out + c] = quantize_one(bf16_to_f32(x[r * ld + c]), scale[axis == 0 ? c : r], fmt, overflow);
+}
+
 /* --------------------------------------------------------------------- GEMM */
 
 /* One output element of D = (A.B) * sa_inv * sb_inv.
@@ -318,6 +373,19 @@ void fp8o_gemm_rows(const uint8_t* A, int fmt_a, int64_t a_si, int64_t a_sk,
         for (int64_t j = 0; j < N; ++j)
             fp8o_gemm_element(A, fmt_a, a_si, a_sk, B, fmt_b, b_sk, b_sj, K, i, j,
                               sa_inv, sb_inv, &ref[(i - i0) * N + j], &sabs[(i - i0) * N + j]);
+}
+
+/* Per-channel weight scales: column j of B (one output channel) carries its own
+ * inverse scale sb_inv_vec[j]; A keeps one per-tensor inverse scale. */
+void fp8o_gemm_rows_colscale(const uint8_t* A, int fmt_a, int64_t a_si, int64_t a_sk,
+                             const uint8_t* B, int fmt_b, int64_t b_sk, int64_t b_sj,
+                             int64_t N, int64_t K, int64_t i0, int64_t i1,
+                             float sa_inv, const float* sb_inv_vec, double* ref, double* sabs)
+{
+    for (int64_t i = i0; i < i1; ++i)
+        for (int64_t j = 0; j < N; ++j)
+            fp8o_gemm_element(A, fmt_a, a_si, a_sk, B, fmt_b, b_sk, b_sj, K, i, j,
+                              sa_inv, sb_inv_vec[j], &ref[(i - i0) * N + j], &sabs[(i - i0) * N + j]);
 }
 
 /* A list of (i,j) samples. */

@@ -111,3 +111,31 @@ def test_special_codes_propagate():
     ref, _ = oracle.gemm_rows(A, E5M2, (K, 1), B, E4M3, (1, 1), 1, K, 0, 1, 1.0, 1.0)
     assert np.isnan(ref[0, 0])
     assert oracle.dot_exact(A[0], E5M2, B[:, 0].copy(), E4M3) is None
+
+
+def test_per_channel_scales_reduce_to_per_tensor_routines():
+    """Section 4.2: per-channel weight scales.  Channel by channel the functions equal the per-tensor
+    ones (pinned separately), and a column-scaled GEMM is the per-tensor GEMM column by column."""
+    rng = np.random.default_rng(40)
+    x = (rng.standard_normal((37, 53)) * np.exp2(rng.uniform(-4, 4, size=(37, 53)))).astype(np.float32)
+    x[5, 7] = np.nan
+    for axis in (0, 1):
+        am = oracle.amax_channels(x, axis)
+        chans = x.T if axis == 0 else x
+        want = np.array([oracle.amax_bits(np.ascontiguousarray(ch)) for ch in chans], dtype=np.uint32)
+        assert np.array_equal(am.view(np.uint32), want)
+        am = np.where(np.isnan(am), 1.0, am).astype(np.float32)
+        s, si = oracle.scales_from_amax(am, E4M3)
+        assert np.array_equal(s, np.float32(448.0) / am)                 # numpy float32 division
+        q = oracle.quantize_channels(x, s, axis, E4M3)
+        for ci, ch in enumerate(chans):
+            got = q[:, ci] if axis == 0 else q[ci]
+            assert np.array_equal(got, oracle.quantize(np.ascontiguousarray(ch), s[ci], E4M3))
+    M, N, K = 6, 9, 40
+    A = _finite_codes(rng, E4M3, (M, K))
+    B = _finite_codes(rng, E4M3, (K, N))
+    sv = np.exp2(rng.uniform(-6, 2, size=N)).astype(np.float32)
+    ref, sab = oracle.gemm_rows_colscale(A, E4M3, (K, 1), B, E4M3, (N, 1), N, K, 0, M, 0.5, sv)
+    for j in range(N):
+        r1, s1 = oracle.gemm_rows(A, E4M3, (K, 1), B, E4M3, (N, 1), N, K, 0, M, 0.5, sv[j])
+        assert np.array_equal(ref[:, j], r1[:, j]) and np.array_equal(sab[:, j], s1[:, j])
