@@ -225,6 +225,37 @@ fp8_status fp8_gemm_fp8out(const fp8_gemm_desc* d, const uint8_t* A, const uint8
                            float* amax_d_dev, void* stream);
 
 /*
+ * Per-channel scale factors — Section 4.2: post-training quantization uses "per-channel scaling factors for
+ * weights, per-tensor scaling factors for activations".  A channel is a row or a column of a 2-D tensor
+ * x (rows x cols, row-major, pitch ld elements): axis 0 = one channel per column, axis 1 = one per row.
+ *
+ * fp8_amax_channels      amax_vec[c] = amax over channel c (definition of fp8_amax), OVERWRITTEN.
+ * fp8_scales_from_amax   `count` scale factors at once, arithmetic of fp8_scale_from_amax; pow2 != 0 gives
+ *                        the power-of-two scales of fp8_scale_pow2_from_amax.
+ * fp8_quantize_channels  out[r*ld_out + c] = encode_f( binary32(x[r*ld + c]) * scale_vec[channel of (r,c)] ),
+ *                        conversion rules of fp8_quantize.
+ * Fast paths need 16-byte aligned rows (base and pitch); anything else takes element-wise kernels with
+ * identical results.
+ */
+fp8_status fp8_amax_channels(const void* x, fp8_wide t, int64_t rows, int64_t cols, int64_t ld, int axis,
+                             float* amax_vec_dev, void* stream);
+fp8_status fp8_scales_from_amax(const float* amax_vec_dev, int64_t count, fp8_format f, int pow2,
+                                float* scale_vec_dev, float* scale_inv_vec_dev, void* stream);
+fp8_status fp8_quantize_channels(const void* x, fp8_wide t, int64_t rows, int64_t cols, int64_t ld, int axis,
+                                 fp8_format f, fp8_overflow o, const float* scale_vec_dev,
+                                 uint8_t* out, int64_t ld_out, void* stream);
+
+/*
+ * fp8_gemm_channel_scales — fp8_gemm for a B operand (the weights) quantized with per-channel scales:
+ *   D[i,j] = round_out( (sum_k decode(A[i,k]) * decode(B[k,j])) * (sa_inv * sb_inv_vec[j]) )
+ * scale_inv_b_vec_dev holds N device floats, one per column j of B (per output channel).  A keeps its
+ * per-tensor inverse scale.  Everything else as fp8_gemm.
+ */
+fp8_status fp8_gemm_channel_scales(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,
+                                   const float* scale_inv_a_dev, const float* scale_inv_b_vec_dev,
+                                   float* amax_d_dev, void* stream);
+
+/*
  * fp8_async_status — reads and clears the device-side error latch of the
  * current device (synchronises the device).  FP8_OK, or FP8_ERR_TIMEOUT if a
  * kernel gave up on a bounded wait since the last call; *detail (optional, host

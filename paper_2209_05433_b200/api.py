@@ -21,7 +21,8 @@ MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
 
 EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
            "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_fake_quantize",
-           "fp8_scale_pow2_from_amax", "fp8_gemm", "fp8_gemm_fp8out",
+           "fp8_scale_pow2_from_amax", "fp8_gemm", "fp8_gemm_fp8out", "fp8_amax_channels", "fp8_scales_from_amax",
+           "fp8_quantize_channels", "fp8_gemm_channel_scales",
            "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
 
 
@@ -80,6 +81,15 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.fp8_gemm_fp8out.restype = i32
     lib.fp8_gemm_fp8out.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+    i64 = ctypes.c_int64
+    lib.fp8_amax_channels.restype = i32
+    lib.fp8_amax_channels.argtypes = [vp, i32, i64, i64, i64, i32, vp, vp]
+    lib.fp8_scales_from_amax.restype = i32
+    lib.fp8_scales_from_amax.argtypes = [vp, i64, i32, i32, vp, vp, vp]
+    lib.fp8_quantize_channels.restype = i32
+    lib.fp8_quantize_channels.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, vp, vp, i64, vp]
+    lib.fp8_gemm_channel_scales.restype = i32
+    lib.fp8_gemm_channel_scales.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.fp8_async_status.restype = i32
     lib.fp8_async_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
     lib.fp8_status_string.restype = ctypes.c_char_p
@@ -240,6 +250,59 @@ def fp8_gemm_fp8out(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int,
                                   _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
                                   _scalar(scale_d, "scale_d"), None if amax_out is None else _scalar(amax_out, "amax_out"),
                                   _stream()), "fp8_gemm_fp8out")
+
+
+def _vec(t: torch.Tensor, count: int, name: str) -> int:
+    if t.dtype != torch.float32 or t.numel() != count:
+        raise TypeError("%s must be a float32 CUDA tensor with %d elements" % (name, count))
+    return _dev(t, name)
+
+
+def _rows2d(t: torch.Tensor, name: str):
+    if t.dim() != 2 or not t.is_cuda or t.stride(1) != 1:
+        raise ValueError("%s must be a 2-D CUDA tensor with unit inner stride" % name)
+    return t.shape[0], t.shape[1], t.stride(0)
+
+
+def fp8_amax_channels(x: torch.Tensor, axis: int, amax_vec: torch.Tensor) -> None:
+    rows, cols, ld = _rows2d(x, "x")
+    _check(load().fp8_amax_channels(x.data_ptr(), _wide_of(x), rows, cols, ld, axis,
+                                    _vec(amax_vec, cols if axis == 0 else rows, "amax_vec"), _stream()), "fp8_amax_channels")
+
+
+def fp8_scales_from_amax(amax_vec: torch.Tensor, fmt: int, scale_vec: torch.Tensor, scale_inv_vec: torch.Tensor, pow2: bool = False) -> None:
+    n = amax_vec.numel()
+    _check(load().fp8_scales_from_amax(_vec(amax_vec, n, "amax_vec"), n, fmt, 1 if pow2 else 0, _vec(scale_vec, n, "scale_vec"),
+                                       _vec(scale_inv_vec, n, "scale_inv_vec"), _stream()), "fp8_scales_from_amax")
+
+
+def fp8_quantize_channels(x: torch.Tensor, axis: int, fmt: int, scale_vec: torch.Tensor, out: torch.Tensor, overflow: int = SATURATE) -> None:
+    rows, cols, ld = _rows2d(x, "x")
+    orows, ocols, ld_out = _rows2d(out, "out")
+    if out.dtype != torch.uint8 or (orows, ocols) != (rows, cols):
+        raise TypeError("out must be a uint8 tensor of the shape of x")
+    _check(load().fp8_quantize_channels(x.data_ptr(), _wide_of(x), rows, cols, ld, axis, fmt, overflow,
+                                        _vec(scale_vec, cols if axis == 0 else rows, "scale_vec"), out.data_ptr(), ld_out, _stream()),
+           "fp8_quantize_channels")
+
+
+def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
+                            scale_inv_a: torch.Tensor, scale_inv_b_vec: torch.Tensor, amax_out: torch.Tensor | None = None) -> None:
+    """fp8_gemm with one inverse scale per column of B (per output channel)."""
+    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
+        raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D tensor")
+    for t, name in ((A, "A"), (B, "B"), (D, "D")):
+        if not t.is_cuda or t.stride(1) != 1:
+            raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
+    M, K = (A.shape[0], A.shape[1]) if ma == MAJOR_K else (A.shape[1], A.shape[0])
+    Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
+    if K != Kb or tuple(D.shape) != (M, N):
+        raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
+    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D))
+    _check(load().fp8_gemm_channel_scales(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
+                                          _scalar(scale_inv_a, "scale_inv_a"), _vec(scale_inv_b_vec, N, "scale_inv_b_vec"),
+                                          None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()),
+           "fp8_gemm_channel_scales")
 
 
 def fp8_async_status() -> tuple[int, int]:

@@ -605,6 +605,217 @@ __global__ void k_scale_pow2_from_amax(const float* amax_dev, float fmax, float*
 }
 
 // ---------------------------------------------------------------------------
+// per-channel scales (Section 4.2: per-channel for weights, per-tensor for activations)
+// x is rows x cols, row-major, pitch ld elements.  AXIS 0: one channel per column; AXIS 1: one per row.
+// ---------------------------------------------------------------------------
+
+// AXIS 0, vector path: a thread owns one 16-byte item of columns (8 bf16 / 4 f32) and walks down a slab of
+// rows; per-column maxima stay separate inside the packed words.  amax_bits[cols] must be zero before.
+template <int WIDE>
+__global__ void __launch_bounds__(kThreads)
+k_amax_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, int64_t rows_per_slab, uint32_t* amax_bits) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
+    const int64_t item = (int64_t)blockIdx.x * kThreads + threadIdx.x;          // item index along the row
+    const int64_t c0 = item * EPI;
+    if (c0 >= cols) return;
+    const int64_t r0 = (int64_t)blockIdx.y * rows_per_slab;
+    const int64_t r1 = min(rows, r0 + rows_per_slab);
+    const char* base = reinterpret_cast<const char*>(x) + c0 * ESZ;
+    uint4 m = make_uint4(0u, 0u, 0u, 0u);
+    auto fold = [&](const uint4& v) {
+        if (WIDE == kWideBF16) {
+            m.x = __vmaxu2(m.x, v.x & 0x7FFF7FFFu); m.y = __vmaxu2(m.y, v.y & 0x7FFF7FFFu);
+            m.z = __vmaxu2(m.z, v.z & 0x7FFF7FFFu); m.w = __vmaxu2(m.w, v.w & 0x7FFF7FFFu);
+        } else {
+            m.x = max(m.x, v.x & 0x7FFFFFFFu); m.y = max(m.y, v.y & 0x7FFFFFFFu);
+            m.z = max(m.z, v.z & 0x7FFFFFFFu); m.w = max(m.w, v.w & 0x7FFFFFFFu);
+        }
+    };
+    int64_t r = r0;
+    for (; r + 4 <= r1; r += 4) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld_nc_v4(base + (r + u) * ld * ESZ);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) fold(v[u]);
+    }
+    for (; r < r1; ++r) fold(ld_nc_v4(base + r * ld * ESZ));
+    const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+    for (int i = 0; i < EPI; ++i) {
+        if (c0 + i < cols) {
+            const uint32_t bits = WIDE == kWideBF16 ? (((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu)) << 16) : w[i];
+            if (bits) atomicMax(&amax_bits[c0 + i], canonical_nan_bits(bits));
+        }
+    }
+}
+
+// AXIS 1, vector path: one warp per row.
+template <int WIDE>
+__global__ void __launch_bounds__(kThreads)
+k_amax_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, uint32_t* amax_bits) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * kThreads) >> 5;
+    const int64_t n_items = cols / EPI;
+    for (int64_t r = warp; r < rows; r += n_warps) {
+        const char* row = reinterpret_cast<const char*>(x) + r * ld * ESZ;
+        uint32_t m = 0;
+        for (int64_t i = lane; i < n_items; i += 32) m = fold_abs_max<WIDE>(m, ld_nc_v4(row + i * 16));
+        m = finish_abs_max<WIDE>(m);
+        for (int64_t c = n_items * EPI + lane; c < cols; c += 32) m = max(m, canonical_nan_bits(scalar_abs_bits<WIDE>(row, c)));
+        m = warp_max_u32(m);
+        if (lane == 0) amax_bits[r] = m;
+    }
+}
+
+// any alignment: one thread per element, channel maxima by atomicMax (amax_bits zero before)
+template <int WIDE, int AXIS>
+__global__ void __launch_bounds__(kThreads)
+k_amax_channels_elementwise(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, uint32_t* amax_bits) {
+    const int64_t total = rows * cols;
+    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kThreads) {
+        const int64_t r = i / cols, c = i - r * cols;
+        const uint32_t bits = canonical_nan_bits(scalar_abs_bits<WIDE>(x, r * ld + c));
+        if (bits) atomicMax(&amax_bits[AXIS == 0 ? c : r], bits);
+    }
+}
+
+// N scaled values with their source sign words -> packed codes (N = 4 or 8)
+template <int FMT, bool NOSAT, int N>
+__device__ __forceinline__ void encode_group(const float (&y)[N], const uint32_t (&xsign)[N], uint32_t (&codes)[N / 4]) {
+    if (!needs_scalar_path<FMT, NOSAT>(y)) {
+#pragma unroll
+        for (int q = 0; q < N / 4; ++q) codes[q] = cvt_quad<FMT>(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+    } else {
+#pragma unroll
+        for (int q = 0; q < N / 4; ++q)
+            codes[q] = encode_scaled<FMT, NOSAT>(y[4 * q], xsign[4 * q]) | (encode_scaled<FMT, NOSAT>(y[4 * q + 1], xsign[4 * q + 1]) << 8) |
+                       (encode_scaled<FMT, NOSAT>(y[4 * q + 2], xsign[4 * q + 2]) << 16) | (encode_scaled<FMT, NOSAT>(y[4 * q + 3], xsign[4 * q + 3]) << 24);
+    }
+}
+
+// one 16-byte item with one scale per element (AXIS 0) -> packed codes
+template <int WIDE, int FMT, bool NOSAT>
+__device__ __forceinline__ void quantize_item_scales(const uint4& v, const float* sc, uint32_t* codes) {
+    if (WIDE == kWideBF16) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        float y[8];
+        uint32_t xs[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            y[2 * i] = __uint_as_float(w[i] << 16) * sc[2 * i];
+            y[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u) * sc[2 * i + 1];
+            xs[2 * i] = w[i] << 16;
+            xs[2 * i + 1] = w[i];
+        }
+        uint32_t c[2];
+        encode_group<FMT, NOSAT, 8>(y, xs, c);
+        codes[0] = c[0]; codes[1] = c[1];
+    } else {
+        float y[4] = {__uint_as_float(v.x) * sc[0], __uint_as_float(v.y) * sc[1], __uint_as_float(v.z) * sc[2], __uint_as_float(v.w) * sc[3]};
+        uint32_t xs[4] = {v.x, v.y, v.z, v.w};
+        uint32_t c[1];
+        encode_group<FMT, NOSAT, 4>(y, xs, c);
+        codes[0] = c[0];
+    }
+}
+
+// AXIS 0, vector path: thread owns one item of columns and its scales, walks down a slab of rows.
+template <int WIDE, int FMT, bool NOSAT>
+__global__ void __launch_bounds__(kThreads)
+k_quantize_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, int64_t rows_per_slab,
+                const float* __restrict__ scale, uint8_t* __restrict__ out, int64_t ld_out) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
+    const int64_t item = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    const int64_t c0 = item * EPI;
+    if (c0 + EPI > cols) return;                                   // ragged right edge: handled by the tail kernel
+    float sc[EPI];
+#pragma unroll
+    for (int i = 0; i < EPI; ++i) sc[i] = __ldg(scale + c0 + i);
+    const int64_t r0 = (int64_t)blockIdx.y * rows_per_slab;
+    const int64_t r1 = min(rows, r0 + rows_per_slab);
+    const char* base = reinterpret_cast<const char*>(x) + c0 * ESZ;
+    for (int64_t r = r0; r < r1; r += 2) {
+        const bool two = r + 1 < r1;
+        const uint4 v0 = ld_nc_v4(base + r * ld * ESZ);
+        const uint4 v1 = two ? ld_nc_v4(base + (r + 1) * ld * ESZ) : v0;
+        uint32_t c[2];
+        quantize_item_scales<WIDE, FMT, NOSAT>(v0, sc, c);
+        if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out + r * ld_out + c0), make_uint2(c[0], c[1]));
+        else                   st_out(reinterpret_cast<uint32_t*>(out + r * ld_out + c0), c[0]);
+        if (two) {
+            quantize_item_scales<WIDE, FMT, NOSAT>(v1, sc, c);
+            if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out + (r + 1) * ld_out + c0), make_uint2(c[0], c[1]));
+            else                   st_out(reinterpret_cast<uint32_t*>(out + (r + 1) * ld_out + c0), c[0]);
+        }
+    }
+}
+
+// AXIS 1, vector path: one warp per row, the row's scale in a register.
+template <int WIDE, int FMT, bool NOSAT>
+__global__ void __launch_bounds__(kThreads)
+k_quantize_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, const float* __restrict__ scale,
+                uint8_t* __restrict__ out, int64_t ld_out) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * kThreads) >> 5;
+    const int64_t n_items = cols / EPI;
+    for (int64_t r = warp; r < rows; r += n_warps) {
+        const float s = __ldg(scale + r);
+        const char* row = reinterpret_cast<const char*>(x) + r * ld * ESZ;
+        uint8_t* orow = out + r * ld_out;
+        for (int64_t i = lane; i < n_items; i += 32) {
+            const uint4 v = ld_nc_v4(row + i * 16);
+            if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(orow) + i, quantize_item_bf16<FMT, NOSAT>(v, s));
+            else                   st_out(reinterpret_cast<uint32_t*>(orow) + i, quantize_item_f32<FMT, NOSAT>(v, s));
+        }
+        for (int64_t c = n_items * EPI + lane; c < cols; c += 32) {
+            const float xf = scalar_load<WIDE>(row, c);
+            orow[c] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * s, __float_as_uint(xf));
+        }
+    }
+}
+
+// any alignment / ragged columns [c_begin, cols): one thread per element
+template <int WIDE, int FMT, bool NOSAT, int AXIS>
+__global__ void __launch_bounds__(kThreads)
+k_quantize_channels_elementwise(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, int64_t c_begin,
+                                const float* __restrict__ scale, uint8_t* __restrict__ out, int64_t ld_out) {
+    const int64_t width = cols - c_begin;
+    const int64_t total = rows * width;
+    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kThreads) {
+        const int64_t r = i / width, c = c_begin + (i - r * width);
+        const float xf = scalar_load<WIDE>(x, r * ld + c);
+        out[r * ld_out + c] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * __ldg(scale + (AXIS == 0 ? c : r)), __float_as_uint(xf));
+    }
+}
+
+// `count` scales at once (per-channel); pow2 != 0 rounds each down to a power of two
+__global__ void __launch_bounds__(kThreads)
+k_scales_from_amax(const float* amax, int64_t count, float fmax, int pow2, float* scale, float* scale_inv) {
+    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < count; i += (int64_t)gridDim.x * kThreads) {
+        float s, si;
+        scale_pair_from_amax(amax[i], fmax, s, si);
+        if (pow2) {
+            uint32_t b = __float_as_uint(s);
+            if ((b >> 23) != 0u) b &= 0x7F800000u;
+            else if (b != 0u) b = 1u << (31 - __clz(b));
+            s = __uint_as_float(b);
+            si = __fdiv_rn(1.0f, s);
+        }
+        scale[i] = s;
+        scale_inv[i] = si;
+    }
+}
+
+// ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
 
@@ -752,6 +963,84 @@ static fp8_status launch_fake(const void* x, size_t n, const float* scale, const
     return launch_status();
 }
 
+static int grid_for(int64_t work_items) {
+    int64_t g = (work_items + kThreads - 1) / kThreads;
+    const int64_t cap = (int64_t)sm_count() * 8;
+    if (g > cap) g = cap;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+// rows per slab so that the 2-D grids of the column kernels fill the machine about four times over
+static int64_t slab_rows(int64_t rows, int64_t col_blocks) {
+    const int64_t want_blocks = (int64_t)sm_count() * 32;
+    int64_t slabs = (want_blocks + col_blocks - 1) / col_blocks;
+    if (slabs < 1) slabs = 1;
+    if (slabs > 65535) slabs = 65535;
+    int64_t per = (rows + slabs - 1) / slabs;
+    per = (per + 3) / 4 * 4;
+    if (per < 4) per = 4;
+    return per;
+}
+
+template <int WIDE>
+static fp8_status launch_amax_channels(const void* x, int64_t rows, int64_t cols, int64_t ld, int axis, uint32_t* bits, cudaStream_t st) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
+    const int64_t channels = axis == 0 ? cols : rows;
+    const bool vec = aligned16(x) && ((ld * ESZ) & 15) == 0;
+    if (axis == 1 && vec) {                                         // every row written exactly once: no zeroing needed
+        k_amax_rows<WIDE><<<grid_for(rows * 32), kThreads, 0, st>>>(x, rows, cols, ld, bits);
+        count_launches(1);
+        return launch_status();
+    }
+    if (cudaMemsetAsync(bits, 0, (size_t)channels * 4, st) != cudaSuccess) return FP8_ERR_CUDA;
+    count_launches(1);
+    if (axis == 0 && vec && cols % EPI == 0) {
+        const int64_t col_blocks = (cols / EPI + kThreads - 1) / kThreads;
+        const int64_t per = slab_rows(rows, col_blocks);
+        dim3 grid((unsigned)col_blocks, (unsigned)((rows + per - 1) / per));
+        k_amax_cols<WIDE><<<grid, kThreads, 0, st>>>(x, rows, cols, ld, per, bits);
+    } else if (axis == 0) {
+        k_amax_channels_elementwise<WIDE, 0><<<grid_for(rows * cols), kThreads, 0, st>>>(x, rows, cols, ld, bits);
+    } else {
+        k_amax_channels_elementwise<WIDE, 1><<<grid_for(rows * cols), kThreads, 0, st>>>(x, rows, cols, ld, bits);
+    }
+    count_launches(1);
+    return launch_status();
+}
+
+template <int WIDE, int FMT, bool NOSAT>
+static fp8_status launch_quantize_channels(const void* x, int64_t rows, int64_t cols, int64_t ld, int axis, const float* scale,
+                                           uint8_t* out, int64_t ld_out, cudaStream_t st) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
+    const bool vec = aligned16(x) && ((ld * ESZ) & 15) == 0 && (reinterpret_cast<uintptr_t>(out) & (EPI - 1)) == 0 && (ld_out % EPI) == 0;
+    if (vec && axis == 1) {
+        k_quantize_rows<WIDE, FMT, NOSAT><<<grid_for(rows * 32), kThreads, 0, st>>>(x, rows, cols, ld, scale, out, ld_out);
+        count_launches(1);
+        return launch_status();
+    }
+    if (vec && axis == 0 && cols >= EPI) {
+        const int64_t full_cols = cols / EPI * EPI;
+        const int64_t col_blocks = (full_cols / EPI + kThreads - 1) / kThreads;
+        const int64_t per = slab_rows(rows, col_blocks);
+        dim3 grid((unsigned)col_blocks, (unsigned)((rows + per - 1) / per));
+        k_quantize_cols<WIDE, FMT, NOSAT><<<grid, kThreads, 0, st>>>(x, rows, full_cols, ld, per, scale, out, ld_out);
+        count_launches(1);
+        if (full_cols < cols) {
+            k_quantize_channels_elementwise<WIDE, FMT, NOSAT, 0><<<grid_for(rows * (cols - full_cols)), kThreads, 0, st>>>(
+                x, rows, cols, ld, full_cols, scale, out, ld_out);
+            count_launches(1);
+        }
+        return launch_status();
+    }
+    if (axis == 0) k_quantize_channels_elementwise<WIDE, FMT, NOSAT, 0><<<grid_for(rows * cols), kThreads, 0, st>>>(x, rows, cols, ld, 0, scale, out, ld_out);
+    else           k_quantize_channels_elementwise<WIDE, FMT, NOSAT, 1><<<grid_for(rows * cols), kThreads, 0, st>>>(x, rows, cols, ld, 0, scale, out, ld_out);
+    count_launches(1);
+    return launch_status();
+}
+
 }  // namespace fp8b200
 
 using namespace fp8b200;
@@ -855,6 +1144,58 @@ void fp8_cast_read_clear_latch(unsigned int out2[2]) {
         const unsigned int zero[2] = {0u, 0u};
         cudaMemcpyToSymbol(fp8b200::g_cast_latch, zero, sizeof(zero));
     }
+}
+
+fp8_status fp8_amax_channels(const void* x, fp8_wide t, int64_t rows, int64_t cols, int64_t ld, int axis,
+                             float* amax_vec_dev, void* stream) {
+    if (!amax_vec_dev || (!x && rows > 0 && cols > 0)) return FP8_ERR_NULL;
+    if ((t != FP8_F32 && t != FP8_BF16) || (axis != 0 && axis != 1)) return FP8_ERR_ENUM;
+    if (rows < 0 || cols < 0 || ld < cols) return FP8_ERR_SHAPE;
+    const int64_t channels = axis == 0 ? cols : rows;
+    if (channels == 0) return FP8_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint32_t* bits = reinterpret_cast<uint32_t*>(amax_vec_dev);
+    if (rows == 0 || cols == 0) {                                   // empty channels: amax 0
+        if (cudaMemsetAsync(bits, 0, (size_t)channels * 4, st) != cudaSuccess) return FP8_ERR_CUDA;
+        count_launches(1);
+        return FP8_OK;
+    }
+    return t == FP8_F32 ? launch_amax_channels<kWideF32>(x, rows, cols, ld, axis, bits, st)
+                        : launch_amax_channels<kWideBF16>(x, rows, cols, ld, axis, bits, st);
+}
+
+fp8_status fp8_scales_from_amax(const float* amax_vec_dev, int64_t count, fp8_format f, int pow2,
+                                float* scale_vec_dev, float* scale_inv_vec_dev, void* stream) {
+    if (count < 0) return FP8_ERR_SHAPE;
+    if (count == 0) return FP8_OK;
+    if (!amax_vec_dev || !scale_vec_dev || !scale_inv_vec_dev) return FP8_ERR_NULL;
+    if (f != FP8_E4M3 && f != FP8_E5M2) return FP8_ERR_ENUM;
+    k_scales_from_amax<<<grid_for(count), kThreads, 0, (cudaStream_t)stream>>>(amax_vec_dev, count, f == FP8_E4M3 ? 448.0f : 57344.0f,
+                                                                               pow2 ? 1 : 0, scale_vec_dev, scale_inv_vec_dev);
+    count_launches(1);
+    return launch_status();
+}
+
+fp8_status fp8_quantize_channels(const void* x, fp8_wide t, int64_t rows, int64_t cols, int64_t ld, int axis, fp8_format f,
+                                 fp8_overflow o, const float* scale_vec_dev, uint8_t* out, int64_t ld_out, void* stream) {
+    if (!scale_vec_dev || ((!x || !out) && rows > 0 && cols > 0)) return FP8_ERR_NULL;
+    if ((t != FP8_F32 && t != FP8_BF16) || (f != FP8_E4M3 && f != FP8_E5M2) || (o != FP8_SATURATE && o != FP8_NOSAT) ||
+        (axis != 0 && axis != 1))
+        return FP8_ERR_ENUM;
+    if (rows < 0 || cols < 0 || ld < cols || ld_out < cols) return FP8_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return FP8_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool nosat = o == FP8_NOSAT;
+    if (t == FP8_F32) {
+        if (f == FP8_E4M3) return nosat ? launch_quantize_channels<kWideF32, kE4M3, true>(x, rows, cols, ld, axis, scale_vec_dev, out, ld_out, st)
+                                        : launch_quantize_channels<kWideF32, kE4M3, false>(x, rows, cols, ld, axis, scale_vec_dev, out, ld_out, st);
+        return nosat ? launch_quantize_channels<kWideF32, kE5M2, true>(x, rows, cols, ld, axis, scale_vec_dev, out, ld_out, st)
+                     : launch_quantize_channels<kWideF32, kE5M2, false>(x, rows, cols, ld, axis, scale_vec_dev, out, ld_out, st);
+    }
+    if (f == FP8_E4M3) return nosat ? launch_quantize_channels<kWideBF16, kE4M3, true>(x, rows, cols, ld, axis, scale_vec_dev, out, ld_out, st)
+                                    : launch_quantize_channels<kWideBF16, kE4M3, false>(x, rows, cols, ld, axis, scale_vec_dev, out, ld_out, st);
+    return nosat ? launch_quantize_channels<kWideBF16, kE5M2, true>(x, rows, cols, ld, axis, scale_vec_dev, out, ld_out, st)
+                 : launch_quantize_channels<kWideBF16, kE5M2, false>(x, rows, cols, ld, axis, scale_vec_dev, out, ld_out, st);
 }
 
 fp8_status fp8_fake_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o,

@@ -248,6 +248,7 @@ struct Params {
     uint32_t idesc;                 // M field set for the CTA group the kernel was built for
     int tiles_m, tiles_n;           // tiles of (128*CG) x 256
     int a_mn, b_mn;                 // operand stored with its M (resp. N) index contiguous
+    const float* sb_inv_vec;        // optional: one inverse scale per column of B (per output channel), N entries
     const float* scale_d;           // FP8 output only: scale applied before the conversion
     int nosat;                      // FP8 output only: non-saturating conversion
 };
@@ -471,7 +472,8 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
     } else {
         // ------------------------------------------------------------ epilogue (each CTA drains its own 128 rows)
         const int q = warp & 3;                                   // TMEM lane quarter this warp may read
-        const float alpha = __ldg(p.sa_inv) * __ldg(p.sb_inv);
+        const float sa_inv = __ldg(p.sa_inv);
+        const float alpha = p.sb_inv_vec ? 0.0f : sa_inv * __ldg(p.sb_inv);
         const float scale_d = (OUT == OUT_E4M3 || OUT == OUT_E5M2) ? __ldg(p.scale_d) : 1.0f;
         uint32_t running = 0;                                     // max of stored magnitude bits (bf16: 16-bit patterns)
         const uint32_t epi_base = ring + SMEM_TILES + (uint32_t)(warp - 2) * 2u * EPI_BUF_BYTES;
@@ -515,8 +517,17 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     tc_ld32(taddr + c * CHUNK + sub * 32, r);
                     tc_wait_ld();
                     float v[32];
+                    if (p.sb_inv_vec) {                       // per-channel weight scales: one alpha per column
+                        const int64_t scol_v = col + sub * 32;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * alpha;
+                        for (int i = 0; i < 32; ++i) {
+                            const float sb = scol_v + i < p.N ? __ldg(p.sb_inv_vec + scol_v + i) : 0.0f;
+                            v[i] = __uint_as_float(r[i]) * (sa_inv * sb);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * alpha;
+                    }
                     uint32_t w[WORDS];                            // this thread's bytes of its row for these 32 columns
                     if (OUT == OUT_F32) {
 #pragma unroll
@@ -680,7 +691,8 @@ static fp8_status dispatch(int out_kind, const CUtensorMap& ma, const CUtensorMa
 
 // Shared body of fp8_gemm and fp8_gemm_fp8out.
 static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D, int out_kind, int nosat,
-                            const float* sa_inv, const float* sb_inv, const float* scale_d, float* amax_d_dev, cudaStream_t st) {
+                            const float* sa_inv, const float* sb_inv, const float* sb_inv_vec, const float* scale_d,
+                            float* amax_d_dev, cudaStream_t st) {
     const int64_t M = d->M, N = d->N, K = d->K;
     if (M < 0 || N < 0 || K < 0) return FP8_ERR_SHAPE;
     const bool a_mn = d->ma == FP8_MAJOR_MN, b_mn = d->mb == FP8_MAJOR_MN;
@@ -729,7 +741,7 @@ static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint
 
     Params p;
     p.M = M; p.N = N; p.K = K; p.ldd = d->ldd; p.D = D;
-    p.sa_inv = sa_inv; p.sb_inv = sb_inv;
+    p.sa_inv = sa_inv; p.sb_inv = sb_inv; p.sb_inv_vec = sb_inv_vec;
     p.amax_bits = reinterpret_cast<uint32_t*>(amax_d_dev);
     p.tiles_m = (int)tiles_m; p.tiles_n = (int)tiles_n;
     p.a_mn = a_mn ? 1 : 0; p.b_mn = b_mn ? 1 : 0;
@@ -758,7 +770,16 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
     using namespace fp8b200::gemm;
     if (!d || !scale_inv_a_dev || !scale_inv_b_dev) return FP8_ERR_NULL;
     if (!desc_enums_ok(d) || (d->out != FP8_F32 && d->out != FP8_BF16)) return FP8_ERR_ENUM;
-    return gemm_impl(d, A, B, D, d->out == FP8_BF16 ? OUT_BF16 : OUT_F32, 0, scale_inv_a_dev, scale_inv_b_dev, nullptr,
+    return gemm_impl(d, A, B, D, d->out == FP8_BF16 ? OUT_BF16 : OUT_F32, 0, scale_inv_a_dev, scale_inv_b_dev, nullptr, nullptr,
+                     amax_d_dev, (cudaStream_t)stream);
+}
+
+fp8_status fp8_gemm_channel_scales(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,
+                                   const float* scale_inv_a_dev, const float* scale_inv_b_vec_dev, float* amax_d_dev, void* stream) {
+    using namespace fp8b200::gemm;
+    if (!d || !scale_inv_a_dev || !scale_inv_b_vec_dev) return FP8_ERR_NULL;
+    if (!desc_enums_ok(d) || (d->out != FP8_F32 && d->out != FP8_BF16)) return FP8_ERR_ENUM;
+    return gemm_impl(d, A, B, D, d->out == FP8_BF16 ? OUT_BF16 : OUT_F32, 0, scale_inv_a_dev, nullptr, scale_inv_b_vec_dev, nullptr,
                      amax_d_dev, (cudaStream_t)stream);
 }
 
@@ -769,7 +790,7 @@ fp8_status fp8_gemm_fp8out(const fp8_gemm_desc* d, const uint8_t* A, const uint8
     if (!d || !scale_inv_a_dev || !scale_inv_b_dev || !scale_d_dev) return FP8_ERR_NULL;
     if (!desc_enums_ok(d) || (fd != FP8_E4M3 && fd != FP8_E5M2) || (od != FP8_SATURATE && od != FP8_NOSAT)) return FP8_ERR_ENUM;
     return gemm_impl(d, A, B, D, fd == FP8_E4M3 ? OUT_E4M3 : OUT_E5M2, od == FP8_NOSAT ? 1 : 0, scale_inv_a_dev, scale_inv_b_dev,
-                     scale_d_dev, amax_d_dev, (cudaStream_t)stream);
+                     nullptr, scale_d_dev, amax_d_dev, (cudaStream_t)stream);
 }
 
 #ifdef FP8_GEMM_PROFILE
