@@ -256,6 +256,21 @@ fp8_status fp8_gemm_channel_scales(const fp8_gemm_desc* d, const uint8_t* A, con
                                    float* amax_d_dev, void* stream);
 
 /*
+ * fp8_gemm_batched — Section 4.2 quantizes "all input tensors to matrix-multiply operations (including
+ * attention batched matrix multiplies)".  `batch` independent products with the same shape, layouts,
+ * formats and per-tensor scales (one scale for the whole batched tensor), in one launch:
+ *   D_b = (A_b . B_b) * (sa_inv * sb_inv),   A_b = A + b*stride_a, B_b = B + b*stride_b, D_b = D + b*stride_d
+ * Strides are in elements of the respective tensor, at least one whole matrix apart, and 16-byte aligned
+ * (in bytes).  amax_d_dev (optional) receives the amax over all batch members.  batch == 0 is a no-op
+ * (amax = 0); batch <= 65535.  Everything else as fp8_gemm.
+ */
+fp8_status fp8_gemm_batched(const fp8_gemm_desc* d, int64_t batch,
+                            const uint8_t* A, int64_t stride_a, const uint8_t* B, int64_t stride_b,
+                            void* D, int64_t stride_d,
+                            const float* scale_inv_a_dev, const float* scale_inv_b_dev,
+                            float* amax_d_dev, void* stream);
+
+/*
  * fp8_async_status — reads and clears the device-side error latch of the
  * current device (synchronises the device).  FP8_OK, or FP8_ERR_TIMEOUT if a
  * kernel gave up on a bounded wait since the last call; *detail (optional, host

@@ -22,7 +22,7 @@ MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
 EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
            "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_fake_quantize",
            "fp8_scale_pow2_from_amax", "fp8_gemm", "fp8_gemm_fp8out", "fp8_amax_channels", "fp8_scales_from_amax",
-           "fp8_quantize_channels", "fp8_gemm_channel_scales",
+           "fp8_quantize_channels", "fp8_gemm_channel_scales", "fp8_gemm_batched",
            "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
 
 
@@ -90,6 +90,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_quantize_channels.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, vp, vp, i64, vp]
     lib.fp8_gemm_channel_scales.restype = i32
     lib.fp8_gemm_channel_scales.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp]
+    lib.fp8_gemm_batched.restype = i32
+    lib.fp8_gemm_batched.argtypes = [ctypes.POINTER(GemmDesc), i64, vp, i64, vp, i64, vp, i64, vp, vp, vp, vp]
     lib.fp8_async_status.restype = i32
     lib.fp8_async_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
     lib.fp8_status_string.restype = ctypes.c_char_p
@@ -303,6 +305,26 @@ def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, 
                                           _scalar(scale_inv_a, "scale_inv_a"), _vec(scale_inv_b_vec, N, "scale_inv_b_vec"),
                                           None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()),
            "fp8_gemm_channel_scales")
+
+
+def fp8_gemm_batched(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
+                     scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, amax_out: torch.Tensor | None = None) -> None:
+    """Batched fp8_gemm: A, B are 3-D uint8 tensors [batch, rows, cols] (layouts per member as fp8_gemm), D is
+    [batch, M, N]; the batch strides are taken from the tensors."""
+    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 3 or B.dim() != 3 or D.dim() != 3:
+        raise TypeError("A and B must be 3-D uint8 tensors and D a 3-D tensor")
+    for t, name in ((A, "A"), (B, "B"), (D, "D")):
+        if not t.is_cuda or t.stride(2) != 1:
+            raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
+    batch = A.shape[0]
+    M, K = (A.shape[1], A.shape[2]) if ma == MAJOR_K else (A.shape[2], A.shape[1])
+    Kb, N = (B.shape[2], B.shape[1]) if mb == MAJOR_K else (B.shape[1], B.shape[2])
+    if K != Kb or B.shape[0] != batch or tuple(D.shape) != (batch, M, N):
+        raise ValueError("shape mismatch")
+    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(1), B.stride(1), D.stride(1), _wide_of(D))
+    _check(load().fp8_gemm_batched(ctypes.byref(d), batch, A.data_ptr(), A.stride(0), B.data_ptr(), B.stride(0),
+                                   D.data_ptr(), D.stride(0), _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
+                                   None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()), "fp8_gemm_batched")
 
 
 def fp8_async_status() -> tuple[int, int]:

@@ -150,10 +150,10 @@ __device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_a
     asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
 }
 // TMA load whose completion is counted on a barrier that may live in the peer CTA of the pair
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t cluster_bar, uint64_t policy) {
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t cluster_bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar), "l"(policy) : "memory");
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(cluster_bar), "l"(policy) : "memory");
 }
 // commit of a CTA-pair MMA: arrives on the barrier at this offset in both CTAs
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
@@ -168,10 +168,10 @@ __device__ __forceinline__ void tc_mma_f8_pair(uint32_t tmem_d, uint64_t adesc, 
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar, uint64_t policy) {
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy) : "memory");
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy) : "memory");
 }
 // L2 eviction policies: operand panels are re-read by many CTAs (keep), the output is written once (stream)
 __device__ __forceinline__ uint64_t policy_evict_last() {
@@ -186,9 +186,9 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
 }
 
 // TMA tensor store of one staged box, tracked by the issuing thread's bulk async-group
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1, uint64_t policy) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
-                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "l"(policy) : "memory");
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], [%1], %5;"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
@@ -248,6 +248,8 @@ struct Params {
     uint32_t idesc;                 // M field set for the CTA group the kernel was built for
     int tiles_m, tiles_n;           // tiles of (128*CG) x 256
     int a_mn, b_mn;                 // operand stored with its M (resp. N) index contiguous
+    int batch;                      // independent problems sharing the scales (strided batch); tiles_m*tiles_n tiles each
+    int64_t stride_d;               // elements between consecutive batch members of D
     const float* sb_inv_vec;        // optional: one inverse scale per column of B (per output channel), N entries
     const float* scale_d;           // FP8 output only: scale applied before the conversion
     int nosat;                      // FP8 output only: non-saturating conversion
@@ -332,7 +334,8 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
     const int lane = threadIdx.x & 31;
     const uint32_t cta_rank = CG == 2 ? cluster_ctarank() : 0u;   // 0 = leader of the pair
     const int worker = blockIdx.x / CG, num_workers = gridDim.x / CG;
-    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int tiles_per_batch = p.tiles_m * p.tiles_n;
+    const int num_tiles = tiles_per_batch * p.batch;
     const int k_blocks = (int)((p.K + BK - 1) / BK);
     const bool A_MN = p.a_mn != 0, B_MN = p.b_mn != 0;
     constexpr int FG = G::FG;
@@ -367,7 +370,8 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         PROF_DECL
         for (int t = worker; t < num_tiles && ok; t += num_workers) {
             int tm, tn;
-            tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
+            const int bi = t / tiles_per_batch;                                 // batch member
+            tile_coords(t - bi * tiles_per_batch, p.tiles_m, p.tiles_n, tm, tn);
             const int m0 = tm * G::TILE_M + (int)cta_rank * BM;                 // this CTA's 128 rows of A
             const int n0 = tn * BN + (int)cta_rank * (BN / CG);                 // this CTA's rows of B
             for (int kb = 0; kb < k_pad; ++kb) {
@@ -384,23 +388,23 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                         const uint32_t full = map_to_cta(pair_bar, 0);                    // the leader's barrier
                         if (kb < k_blocks) {
                             mbar_arrive_expect_tx_cluster(full, STAGE_BYTES);
-                            if (A_MN) tma_load_2d_pair(sa, &map_a, m0, k0, full, keep);     // box {128 m, 128 k}
-                            else      tma_load_2d_pair(sa, &map_a, k0, m0, full, keep);     // box {128 k, 128 m}
-                            if (B_MN) tma_load_2d_pair(sb, &map_b, n0, k0, full, keep);     // box {128 n, 128 k}
-                            else      tma_load_2d_pair(sb, &map_b, k0, n0, full, keep);     // box {128 k, 128 n}
+                            if (A_MN) tma_load_3d_pair(sa, &map_a, m0, k0, bi, full, keep);     // box {128 m, 128 k}
+                            else      tma_load_3d_pair(sa, &map_a, k0, m0, bi, full, keep);     // box {128 k, 128 m}
+                            if (B_MN) tma_load_3d_pair(sb, &map_b, n0, k0, bi, full, keep);     // box {128 n, 128 k}
+                            else      tma_load_3d_pair(sb, &map_b, k0, n0, bi, full, keep);     // box {128 k, 128 n}
                         } else {
                             mbar_arrive_cluster(full);                                    // padding block: nothing to load
                         }
                     } else {
                         if (kb < k_blocks) {
                             mbar_arrive_expect_tx(pair_bar, STAGE_BYTES);
-                            if (A_MN) tma_load_2d(sa, &map_a, m0, k0, pair_bar, keep);
-                            else      tma_load_2d(sa, &map_a, k0, m0, pair_bar, keep);
+                            if (A_MN) tma_load_3d(sa, &map_a, m0, k0, bi, pair_bar, keep);
+                            else      tma_load_3d(sa, &map_a, k0, m0, bi, pair_bar, keep);
                             if (B_MN) {                                               // two boxes {128 n, 128 k}
-                                tma_load_2d(sb, &map_b, n0, k0, pair_bar, keep);
-                                tma_load_2d(sb + G::B_BYTES / 2, &map_b, n0 + 128, k0, pair_bar, keep);
+                                tma_load_3d(sb, &map_b, n0, k0, bi, pair_bar, keep);
+                                tma_load_3d(sb + G::B_BYTES / 2, &map_b, n0 + 128, k0, bi, pair_bar, keep);
                             } else {
-                                tma_load_2d(sb, &map_b, k0, n0, pair_bar, keep);        // box {128 k, 256 n}
+                                tma_load_3d(sb, &map_b, k0, n0, bi, pair_bar, keep);        // box {128 k, 256 n}
                             }
                         } else {
                             mbar_arrive(pair_bar);
@@ -484,7 +488,8 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         PROF_DECL
         for (int t = worker; t < num_tiles && ok; t += num_workers, ++it) {
             int tm, tn;
-            tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
+            const int bi = t / tiles_per_batch;
+            tile_coords(t - bi * tiles_per_batch, p.tiles_m, p.tiles_n, tm, tn);
             const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
             PROF_BEGIN
             ok = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, WAIT_ACC_FULL);
@@ -563,7 +568,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     }
                     if (direct) {
                         if (row_ok) {
-                            uint8_t* drow = reinterpret_cast<uint8_t*>(p.D) + (((int64_t)row0 + lane) * p.ldd + scol) * ESZ;
+                            uint8_t* drow = reinterpret_cast<uint8_t*>(p.D) + ((int64_t)bi * p.stride_d + ((int64_t)row0 + lane) * p.ldd + scol) * ESZ;
                             for (int i = 0; i < 32 && scol + i < p.N; ++i) {
                                 if (OUT == OUT_F32)       reinterpret_cast<uint32_t*>(drow)[i] = w[i];
                                 else if (OUT == OUT_BF16) reinterpret_cast<uint16_t*>(drow)[i] = (uint16_t)((i & 1) ? (w[i >> 1] >> 16) : w[i >> 1]);
@@ -583,7 +588,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    if (row0 < p.M && col < p.N) tma_store_2d(&map_d, sbuf, (int)(col * ESZ), row0, stream_out);
+                    if (row0 < p.M && col < p.N) tma_store_3d(&map_d, sbuf, (int)(col * ESZ), row0, bi, stream_out);
                     bulk_commit();
                 }
                 buf ^= 1u;
@@ -633,16 +638,17 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// 2-D byte tensor {inner, outer} with row pitch `pitch`, box {box_inner, box_outer}, 128B swizzle, zero fill.
+// 3-D byte tensor {inner, outer, batch} with row pitch `pitch` and batch pitch `batch_pitch` (bytes),
+// box {box_inner, box_outer, 1}, 128B swizzle, zero fill.
 static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch,
-                     uint32_t box_inner, uint32_t box_outer) {
+                     uint64_t batch, uint64_t batch_pitch, uint32_t box_inner, uint32_t box_outer) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {inner, outer};
-    const cuuint64_t strides[1] = {pitch};
-    const cuuint32_t box[2] = {box_inner, box_outer};
-    const cuuint32_t elem[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
+    const cuuint64_t dims[3] = {inner, outer, batch};
+    const cuuint64_t strides[2] = {pitch, batch > 1 ? batch_pitch : pitch * outer};
+    const cuuint32_t box[3] = {box_inner, box_outer, 1};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, elem,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -690,11 +696,13 @@ static fp8_status dispatch(int out_kind, const CUtensorMap& ma, const CUtensorMa
 }
 
 // Shared body of fp8_gemm and fp8_gemm_fp8out.
+struct Batch { int64_t count, stride_a, stride_b, stride_d; };      // strides in elements
+
 static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D, int out_kind, int nosat,
                             const float* sa_inv, const float* sb_inv, const float* sb_inv_vec, const float* scale_d,
-                            float* amax_d_dev, cudaStream_t st) {
+                            float* amax_d_dev, cudaStream_t st, Batch bt = Batch{1, 0, 0, 0}) {
     const int64_t M = d->M, N = d->N, K = d->K;
-    if (M < 0 || N < 0 || K < 0) return FP8_ERR_SHAPE;
+    if (M < 0 || N < 0 || K < 0 || bt.count < 0) return FP8_ERR_SHAPE;
     const bool a_mn = d->ma == FP8_MAJOR_MN, b_mn = d->mb == FP8_MAJOR_MN;
     const int64_t esz = out_kind == OUT_F32 ? 4 : out_kind == OUT_BF16 ? 2 : 1;
     // CTA pairs (256-row tiles) unless the whole problem has at most 128 rows
@@ -712,8 +720,13 @@ static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint
                 return FP8_ERR_ALIGN;
         }
         if ((reinterpret_cast<uintptr_t>(D) & 15u) || ((d->ldd * esz) & 15)) return FP8_ERR_ALIGN;
-        if (tiles_m * tiles_n > (int64_t)1 << 30 || M > ((int64_t)1 << 31) - 256 || N > ((int64_t)1 << 31) - 512 ||
-            K > ((int64_t)1 << 31) - 256)
+        if (bt.count > 1) {
+            const int64_t a_rows = a_mn ? K : M, b_rows_total = b_mn ? K : N;
+            if (bt.stride_a < a_rows * d->lda || bt.stride_b < b_rows_total * d->ldb || bt.stride_d < M * d->ldd) return FP8_ERR_SHAPE;
+            if ((bt.stride_a & 15) || (bt.stride_b & 15) || ((bt.stride_d * esz) & 15)) return FP8_ERR_ALIGN;
+        }
+        if (tiles_m * tiles_n * (bt.count > 0 ? bt.count : 1) > (int64_t)1 << 30 || M > ((int64_t)1 << 31) - 256 ||
+            N > ((int64_t)1 << 31) - 512 || K > ((int64_t)1 << 31) - 256 || bt.count > 65535)
             return FP8_ERR_UNSUPPORTED;
     }
     // ---- work
@@ -721,22 +734,27 @@ static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint
         if (cudaMemsetAsync(amax_d_dev, 0, 4, st) != cudaSuccess) return FP8_ERR_CUDA;
         count_launches(1);
     }
-    if (M == 0 || N == 0) return FP8_OK;
+    if (M == 0 || N == 0 || bt.count == 0) return FP8_OK;
     if (K == 0) {                                                 // empty sum: zeros in every output type
-        if (cudaMemset2DAsync(D, (size_t)(d->ldd * esz), 0, (size_t)(N * esz), (size_t)M, st) != cudaSuccess) return FP8_ERR_CUDA;
-        count_launches(1);
+        for (int64_t b = 0; b < bt.count; ++b) {
+            if (cudaMemset2DAsync(reinterpret_cast<uint8_t*>(D) + b * bt.stride_d * esz, (size_t)(d->ldd * esz), 0, (size_t)(N * esz),
+                                  (size_t)M, st) != cudaSuccess)
+                return FP8_ERR_CUDA;
+            count_launches(1);
+        }
         return FP8_OK;
     }
 
     CUtensorMap map_a, map_b;
     const uint32_t b_rows = (uint32_t)(BN / cg);                  // B rows one CTA loads per K-block
-    bool ok = a_mn ? make_map(&map_a, A, (uint64_t)M, (uint64_t)K, (uint64_t)d->lda, 128, BK)
-                   : make_map(&map_a, A, (uint64_t)K, (uint64_t)M, (uint64_t)d->lda, BK, BM);
-    ok = ok && (b_mn ? make_map(&map_b, B, (uint64_t)N, (uint64_t)K, (uint64_t)d->ldb, 128, BK)
-                     : make_map(&map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)d->ldb, BK, b_rows));
+    const uint64_t nb = (uint64_t)bt.count;
+    bool ok = a_mn ? make_map(&map_a, A, (uint64_t)M, (uint64_t)K, (uint64_t)d->lda, nb, (uint64_t)bt.stride_a, 128, BK)
+                   : make_map(&map_a, A, (uint64_t)K, (uint64_t)M, (uint64_t)d->lda, nb, (uint64_t)bt.stride_a, BK, BM);
+    ok = ok && (b_mn ? make_map(&map_b, B, (uint64_t)N, (uint64_t)K, (uint64_t)d->ldb, nb, (uint64_t)bt.stride_b, 128, BK)
+                     : make_map(&map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)d->ldb, nb, (uint64_t)bt.stride_b, BK, b_rows));
     // D as a byte tensor {N*esz, M}: boxes of 128 bytes x 32 rows, the unit each epilogue warp stores
     CUtensorMap map_d;
-    ok = ok && make_map(&map_d, D, (uint64_t)(N * esz), (uint64_t)M, (uint64_t)(d->ldd * esz), 128, 32);
+    ok = ok && make_map(&map_d, D, (uint64_t)(N * esz), (uint64_t)M, (uint64_t)(d->ldd * esz), nb, (uint64_t)(bt.stride_d * esz), 128, 32);
     if (!ok) return FP8_ERR_CUDA;
 
     Params p;
@@ -745,12 +763,13 @@ static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint
     p.amax_bits = reinterpret_cast<uint32_t*>(amax_d_dev);
     p.tiles_m = (int)tiles_m; p.tiles_n = (int)tiles_n;
     p.a_mn = a_mn ? 1 : 0; p.b_mn = b_mn ? 1 : 0;
+    p.batch = (int)bt.count; p.stride_d = bt.stride_d;
     p.scale_d = scale_d; p.nosat = nosat;
     // instruction descriptor: fp32 accumulate, operand formats and majors, N/8, M/16 (M = 256 for a CTA pair)
     p.idesc = (1u << 4) | ((uint32_t)d->fa << 7) | ((uint32_t)d->fb << 10) | ((a_mn ? 1u : 0u) << 15) |
               ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
-    return cg == 2 ? dispatch<2>(out_kind, map_a, map_b, map_d, p, tiles_m * tiles_n, st)
-                   : dispatch<1>(out_kind, map_a, map_b, map_d, p, tiles_m * tiles_n, st);
+    return cg == 2 ? dispatch<2>(out_kind, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st)
+                   : dispatch<1>(out_kind, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st);
 }
 
 }  // namespace gemm
@@ -772,6 +791,16 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
     if (!desc_enums_ok(d) || (d->out != FP8_F32 && d->out != FP8_BF16)) return FP8_ERR_ENUM;
     return gemm_impl(d, A, B, D, d->out == FP8_BF16 ? OUT_BF16 : OUT_F32, 0, scale_inv_a_dev, scale_inv_b_dev, nullptr, nullptr,
                      amax_d_dev, (cudaStream_t)stream);
+}
+
+fp8_status fp8_gemm_batched(const fp8_gemm_desc* d, int64_t batch, const uint8_t* A, int64_t stride_a, const uint8_t* B, int64_t stride_b,
+                            void* D, int64_t stride_d, const float* scale_inv_a_dev, const float* scale_inv_b_dev,
+                            float* amax_d_dev, void* stream) {
+    using namespace fp8b200::gemm;
+    if (!d || !scale_inv_a_dev || !scale_inv_b_dev) return FP8_ERR_NULL;
+    if (!desc_enums_ok(d) || (d->out != FP8_F32 && d->out != FP8_BF16)) return FP8_ERR_ENUM;
+    return gemm_impl(d, A, B, D, d->out == FP8_BF16 ? OUT_BF16 : OUT_F32, 0, scale_inv_a_dev, scale_inv_b_dev, nullptr, nullptr,
+                     amax_d_dev, (cudaStream_t)stream, Batch{batch, stride_a, stride_b, stride_d});
 }
 
 fp8_status fp8_gemm_channel_scales(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,

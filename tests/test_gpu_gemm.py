@@ -288,3 +288,47 @@ def test_fp8_output_special_values_and_k0():
     A0 = torch.empty((64, 0), dtype=torch.uint8, device=DEV)
     api.fp8_gemm_fp8out(A0, E4, api.MAJOR_K, A0, E4, api.MAJOR_K, D, E4, _scalar(1.0), _scalar(1.0), _scalar(1.0), amax)
     assert bool((D == 0).all()) and amax.item() == 0.0
+
+
+# ------------------------------------------------------ batched (attention-style) products --
+
+@pytest.mark.parametrize("case", ["scores", "context", "ragged"])
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_batched_gemm(case, out_dtype):
+    """the two attention products: scores = Q.K^T (both operands K-major, K = head dim) and
+    context = P.V (V stored [S, d]: N contiguous), batch = heads; plus a ragged case with padded pitches"""
+    rng = np.random.default_rng({"scores": 1, "context": 2, "ragged": 3}[case])
+    if case == "scores":
+        batch, M, N, K, ma, mb = 6, 320, 320, 128, api.MAJOR_K, api.MAJOR_K
+    elif case == "context":
+        batch, M, N, K, ma, mb = 5, 256, 128, 384, api.MAJOR_K, api.MAJOR_MN
+    else:
+        batch, M, N, K, ma, mb = 3, 130, 72, 100, api.MAJOR_MN, api.MAJOR_K
+    a_shape = (M, K) if ma == api.MAJOR_K else (K, M)
+    b_shape = (N, K) if mb == api.MAJOR_K else (K, N)
+    A_np = np.stack([_pad_cols(_codes(rng, E4, a_shape)) for _ in range(batch)])
+    B_np = np.stack([_pad_cols(_codes(rng, E4, b_shape)) for _ in range(batch)])
+    A = torch.from_numpy(A_np).to(DEV)[:, :, : a_shape[1]]
+    B = torch.from_numpy(B_np).to(DEV)[:, :, : b_shape[1]]
+    esz = 2 if out_dtype == torch.bfloat16 else 4
+    ldd = (N * esz + 15) // 16 * 16 // esz
+    D_full = torch.full((batch, M + 1, ldd), 777.0, dtype=out_dtype, device=DEV)
+    D = D_full[:, :M, :N]
+    amax = _scalar(-1.0)
+    api.fp8_gemm_batched(A, E4, ma, B, E4, mb, D, _scalar(0.25), _scalar(0.5), amax)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    assert bool((D_full[:, M:, :] == 777.0).all()) and bool((D_full[:, :M, N:] == 777.0).all()), "wrote outside D"
+    a_str = (A_np.shape[2], 1) if ma == api.MAJOR_K else (1, A_np.shape[2])
+    b_str = (1, B_np.shape[2]) if mb == api.MAJOR_K else (B_np.shape[2], 1)
+    got = to_np_bits(D)
+    for b in range(batch):
+        ref, sabs = oracle.gemm_rows(A_np[b], E4, a_str, B_np[b], E4, b_str, N, K, 0, M, 0.25, 0.5, threads=THREADS)
+        if out_dtype == torch.float32:
+            ok, worst = check_gemm_f32(got[b], ref, sabs)
+        else:
+            ok, _ = check_gemm_bf16(got[b], ref, sabs, oracle.round_bf16_from_f64)
+        assert ok.all(), (b, np.argwhere(~ok)[:4].tolist())
+    a2 = _scalar(-1.0)
+    api.fp8_amax(D.contiguous(), a2)
+    assert amax.cpu().numpy().view(np.uint32)[0] == a2.cpu().numpy().view(np.uint32)[0]
