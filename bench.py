@@ -229,6 +229,73 @@ def bench_cast_sweep(torch, api, synth, device, log2n, iters=5):
     return out
 
 
+def bench_next_rows(torch, api, synth, device, pk, iters=5):
+    """The rows beyond the core path, each timed alone on workload-shaped tensors: simulated-FP8 round trip,
+    per-channel weight scales, FP8-output GEMM, attention-style batched GEMM."""
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        times = []
+        for _ in range(iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        return statistics.median(times)
+
+    out = {}
+    f32 = torch.float32
+    sc = torch.tensor([3.0, 1.0 / 3.0, 0.0, 0.0], dtype=f32, device=device)
+    s, si, a = sc[0:1], sc[1:2], sc[2:3]
+    # simulated FP8 (quantize + dequantize in one pass), 2^28 bf16 elements: 4 B per element
+    n = 1 << 28
+    x = synth.normal_laplace_mixture(n, 1, synth.T_ID, device=device)
+    y = torch.empty_like(x)
+    ms = timed(lambda: api.fp8_fake_quantize(x, api.E4M3, s, si, y))
+    out["fake_quantize_e4m3_2pow28"] = {"ms": round(ms, 4), "gbs": round(4.0 * n / ms / 1e6, 1), "frac_of_measured_hbm": round(4.0 * n / ms / 1e6 / pk["hbm_gbs"], 4)}
+    del x, y
+    # per-channel weight scales on W [4096 x 16384] bf16, one channel per output column
+    W = synth.weights(D_IN * D_OUT, 3, W_SIGMA, device=device).view(D_IN, D_OUT)
+    am = torch.empty(D_OUT, dtype=f32, device=device)
+    sv, siv = torch.empty(D_OUT, dtype=f32, device=device), torch.empty(D_OUT, dtype=f32, device=device)
+    Wq = torch.empty(D_IN, D_OUT, dtype=torch.uint8, device=device)
+    nW = D_IN * D_OUT
+    ms = timed(lambda: api.fp8_amax_channels(W, 0, am))
+    out["amax_channels_cols_W"] = {"ms": round(ms, 4), "gbs": round(2.0 * nW / ms / 1e6, 1), "frac_of_measured_hbm": round(2.0 * nW / ms / 1e6 / pk["hbm_gbs"], 4)}
+    api.fp8_scales_from_amax(am, api.E4M3, sv, siv)
+    ms = timed(lambda: api.fp8_quantize_channels(W, 0, api.E4M3, sv, Wq))
+    out["quantize_channels_cols_W"] = {"ms": round(ms, 4), "gbs": round(3.0 * nW / ms / 1e6, 1), "frac_of_measured_hbm": round(3.0 * nW / ms / 1e6 / pk["hbm_gbs"], 4)}
+    # forward GEMM with per-channel weight scales, and with FP8 (E4M3) output
+    X = synth.activations(TOKENS * D_IN, 3, device=device).view(TOKENS, D_IN)
+    Xq = torch.empty(TOKENS, D_IN, dtype=torch.uint8, device=device)
+    sx = torch.zeros(3, dtype=f32, device=device)
+    api.fp8_quantize_current(X, api.E4M3, Xq, sx[0:1], sx[1:2], sx[2:3])
+    Y = torch.empty(TOKENS, D_OUT, dtype=torch.bfloat16, device=device)
+    Yq = torch.empty(TOKENS, D_OUT, dtype=torch.uint8, device=device)
+    flops = 2.0 * TOKENS * D_IN * D_OUT
+    ms = timed(lambda: api.fp8_gemm_channel_scales(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, sx[2:3], siv, a))
+    out["gemm_fprop_channel_scales"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
+    ms = timed(lambda: api.fp8_gemm_fp8out(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Yq, api.E4M3, sx[2:3], si, s, a))
+    out["gemm_fprop_fp8_output"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
+    del W, X, Y, Yq
+    # attention-style batched products: 32 heads, 4096 tokens, head dim 128: scores = Q.K^T, context = P.V
+    H, S, Dh = 32, 4096, 128
+    Q = torch.randint(0, 0x78, (H, S, Dh), dtype=torch.uint8, device=device)
+    Kt = torch.randint(0, 0x78, (H, S, Dh), dtype=torch.uint8, device=device)
+    P = torch.empty(H, S, S, dtype=torch.bfloat16, device=device)
+    ms = timed(lambda: api.fp8_gemm_batched(Q, api.E4M3, api.MAJOR_K, Kt, api.E4M3, api.MAJOR_K, P, si, si, a))
+    fl = 2.0 * H * S * S * Dh
+    out["batched_scores_32x4096x4096x128"] = {"ms": round(ms, 4), "tflops": round(fl / ms / 1e9, 1),
+                                              "output_gbs": round(2.0 * H * S * S / ms / 1e6, 1), "bound": "hbm (bf16 output, K = 128)"}
+    Pq = torch.randint(0, 0x78, (H, S, S), dtype=torch.uint8, device=device)
+    C = torch.empty(H, S, Dh, dtype=torch.bfloat16, device=device)
+    ms = timed(lambda: api.fp8_gemm_batched(Pq, api.E4M3, api.MAJOR_K, Kt, api.E4M3, api.MAJOR_MN, C, si, si, a))
+    out["batched_context_32x4096x128x4096"] = {"ms": round(ms, 4), "tflops": round(fl / ms / 1e9, 1)}
+    del Q, Kt, P, Pq, C
+    torch.cuda.empty_cache()
+    return out
+
+
 # ----------------------------------------------------------------------------
 # the oracle arm (CPU)
 # ----------------------------------------------------------------------------
@@ -438,6 +505,9 @@ def run_ours(args):
             cast = bench_cast_sweep(torch, api, synth, device, args.cast_log2n)
             for v in cast.values():
                 v["frac_of_measured_hbm"] = round(v["gbs"] / pk["hbm_gbs"], 4)
+        next_rows = None
+        if world == 1 and not args.no_next_rows:
+            next_rows = bench_next_rows(torch, api, synth, device, pk)
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
             threads = os.cpu_count() or 1
@@ -455,6 +525,7 @@ def run_ours(args):
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
             "gpu_launches": int(launches), "gpu_launches_note": "kernels plus 4-byte memset nodes enqueued by the library in the timed region",
             "roofline": roofline, "roofline_cast": roofline_cast, "kernels": kernels, "cast_sweep_2pow%d" % args.cast_log2n: cast,
+            "next_rows": next_rows,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
@@ -471,6 +542,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cast-sweep", action="store_true")
+    ap.add_argument("--no-next-rows", action="store_true")
     ap.add_argument("--cast-log2n", type=int, default=28)
     ap.add_argument("--unfused-cast", action="store_true", help="amax, scale and quantize as three calls per tensor instead of fp8_quantize_current")
     ap.add_argument("--only", default=None, help="profiling aid: time only the calls with this label (e.g. gemm_fprop, quantize, amax)")

@@ -609,16 +609,20 @@ __global__ void k_scale_pow2_from_amax(const float* amax_dev, float fmax, float*
 // x is rows x cols, row-major, pitch ld elements.  AXIS 0: one channel per column; AXIS 1: one per row.
 // ---------------------------------------------------------------------------
 
-// AXIS 0, vector path: a thread owns one 16-byte item of columns (8 bf16 / 4 f32) and walks down a slab of
-// rows; per-column maxima stay separate inside the packed words.  amax_bits[cols] must be zero before.
+// AXIS 0, vector path.  Block = 64 items wide x 4 row lanes: a thread owns one 16-byte item of columns
+// (8 bf16 / 4 f32) and every fourth row of the block's slab; per-column maxima stay separate inside the
+// packed words.  The four row lanes meet in shared memory, then one atomicMax per column per block.
+// amax_bits[cols] must be zero before.
+constexpr int kColsTx = 64, kColsTy = 4;
 template <int WIDE>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kColsTx * kColsTy)
 k_amax_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, int64_t rows_per_slab, uint32_t* amax_bits) {
+    __shared__ uint4 part[kColsTy][kColsTx];
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
     constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
-    const int64_t item = (int64_t)blockIdx.x * kThreads + threadIdx.x;          // item index along the row
-    const int64_t c0 = item * EPI;
-    if (c0 >= cols) return;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int64_t c0 = ((int64_t)blockIdx.x * kColsTx + tx) * EPI;
+    const bool live = c0 < cols;
     const int64_t r0 = (int64_t)blockIdx.y * rows_per_slab;
     const int64_t r1 = min(rows, r0 + rows_per_slab);
     const char* base = reinterpret_cast<const char*>(x) + c0 * ESZ;
@@ -632,21 +636,33 @@ k_amax_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, 
             m.z = max(m.z, v.z & 0x7FFFFFFFu); m.w = max(m.w, v.w & 0x7FFFFFFFu);
         }
     };
-    int64_t r = r0;
-    for (; r + 4 <= r1; r += 4) {
-        uint4 v[4];
+    if (live) {
+        int64_t r = r0 + ty;
+        for (; r + 3 * kColsTy < r1; r += 4 * kColsTy) {
+            uint4 v[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = ld_nc_v4(base + (r + u) * ld * ESZ);
+            for (int u = 0; u < 4; ++u) v[u] = ld_nc_v4(base + (r + u * kColsTy) * ld * ESZ);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) fold(v[u]);
+            for (int u = 0; u < 4; ++u) fold(v[u]);
+        }
+        for (; r < r1; r += kColsTy) fold(ld_nc_v4(base + r * ld * ESZ));
     }
-    for (; r < r1; ++r) fold(ld_nc_v4(base + r * ld * ESZ));
-    const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+    part[ty][tx] = m;
+    __syncthreads();
+    if (ty == 0 && live) {
 #pragma unroll
-    for (int i = 0; i < EPI; ++i) {
-        if (c0 + i < cols) {
-            const uint32_t bits = WIDE == kWideBF16 ? (((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu)) << 16) : w[i];
-            if (bits) atomicMax(&amax_bits[c0 + i], canonical_nan_bits(bits));
+        for (int k = 1; k < kColsTy; ++k) {
+            const uint4 o = part[k][tx];
+            if (WIDE == kWideBF16) { m.x = __vmaxu2(m.x, o.x); m.y = __vmaxu2(m.y, o.y); m.z = __vmaxu2(m.z, o.z); m.w = __vmaxu2(m.w, o.w); }
+            else                   { m.x = max(m.x, o.x); m.y = max(m.y, o.y); m.z = max(m.z, o.z); m.w = max(m.w, o.w); }
+        }
+        const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+        for (int i = 0; i < EPI; ++i) {
+            if (c0 + i < cols) {
+                const uint32_t bits = WIDE == kWideBF16 ? (((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu)) << 16) : w[i];
+                if (bits) atomicMax(&amax_bits[c0 + i], canonical_nan_bits(bits));
+            }
         }
     }
 }
@@ -724,15 +740,15 @@ __device__ __forceinline__ void quantize_item_scales(const uint4& v, const float
     }
 }
 
-// AXIS 0, vector path: thread owns one item of columns and its scales, walks down a slab of rows.
+// AXIS 0, vector path.  Same 64 x 4 block shape as k_amax_cols: a thread keeps the scales of its item of
+// columns in registers and converts every fourth row of the slab, four loads in flight.
 template <int WIDE, int FMT, bool NOSAT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kColsTx * kColsTy)
 k_quantize_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, int64_t rows_per_slab,
                 const float* __restrict__ scale, uint8_t* __restrict__ out, int64_t ld_out) {
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
     constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
-    const int64_t item = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    const int64_t c0 = item * EPI;
+    const int64_t c0 = ((int64_t)blockIdx.x * kColsTx + threadIdx.x) * EPI;
     if (c0 + EPI > cols) return;                                   // ragged right edge: handled by the tail kernel
     float sc[EPI];
 #pragma unroll
@@ -740,20 +756,21 @@ k_quantize_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t 
     const int64_t r0 = (int64_t)blockIdx.y * rows_per_slab;
     const int64_t r1 = min(rows, r0 + rows_per_slab);
     const char* base = reinterpret_cast<const char*>(x) + c0 * ESZ;
-    for (int64_t r = r0; r < r1; r += 2) {
-        const bool two = r + 1 < r1;
-        const uint4 v0 = ld_nc_v4(base + r * ld * ESZ);
-        const uint4 v1 = two ? ld_nc_v4(base + (r + 1) * ld * ESZ) : v0;
+    auto emit = [&](int64_t r, const uint4& v) {
         uint32_t c[2];
-        quantize_item_scales<WIDE, FMT, NOSAT>(v0, sc, c);
+        quantize_item_scales<WIDE, FMT, NOSAT>(v, sc, c);
         if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out + r * ld_out + c0), make_uint2(c[0], c[1]));
         else                   st_out(reinterpret_cast<uint32_t*>(out + r * ld_out + c0), c[0]);
-        if (two) {
-            quantize_item_scales<WIDE, FMT, NOSAT>(v1, sc, c);
-            if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out + (r + 1) * ld_out + c0), make_uint2(c[0], c[1]));
-            else                   st_out(reinterpret_cast<uint32_t*>(out + (r + 1) * ld_out + c0), c[0]);
-        }
+    };
+    int64_t r = r0 + threadIdx.y;
+    for (; r + 3 * kColsTy < r1; r += 4 * kColsTy) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld_nc_v4(base + (r + u * kColsTy) * ld * ESZ);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) emit(r + u * kColsTy, v[u]);
     }
+    for (; r < r1; r += kColsTy) emit(r, ld_nc_v4(base + r * ld * ESZ));
 }
 
 // AXIS 1, vector path: one warp per row, the row's scale in a register.
@@ -971,15 +988,15 @@ static int grid_for(int64_t work_items) {
     return (int)g;
 }
 
-// rows per slab so that the 2-D grids of the column kernels fill the machine about four times over
+// rows per slab of the column kernels: about 16 blocks per SM in all, at least 64 rows (16 per thread)
 static int64_t slab_rows(int64_t rows, int64_t col_blocks) {
-    const int64_t want_blocks = (int64_t)sm_count() * 32;
+    const int64_t want_blocks = (int64_t)sm_count() * 16;
     int64_t slabs = (want_blocks + col_blocks - 1) / col_blocks;
     if (slabs < 1) slabs = 1;
-    if (slabs > 65535) slabs = 65535;
     int64_t per = (rows + slabs - 1) / slabs;
-    per = (per + 3) / 4 * 4;
-    if (per < 4) per = 4;
+    per = (per + 15) / 16 * 16;
+    if (per < 64) per = 64;
+    while ((rows + per - 1) / per > 65535) per *= 2;
     return per;
 }
 
@@ -997,10 +1014,10 @@ static fp8_status launch_amax_channels(const void* x, int64_t rows, int64_t cols
     if (cudaMemsetAsync(bits, 0, (size_t)channels * 4, st) != cudaSuccess) return FP8_ERR_CUDA;
     count_launches(1);
     if (axis == 0 && vec && cols % EPI == 0) {
-        const int64_t col_blocks = (cols / EPI + kThreads - 1) / kThreads;
+        const int64_t col_blocks = (cols / EPI + kColsTx - 1) / kColsTx;
         const int64_t per = slab_rows(rows, col_blocks);
         dim3 grid((unsigned)col_blocks, (unsigned)((rows + per - 1) / per));
-        k_amax_cols<WIDE><<<grid, kThreads, 0, st>>>(x, rows, cols, ld, per, bits);
+        k_amax_cols<WIDE><<<grid, dim3(kColsTx, kColsTy), 0, st>>>(x, rows, cols, ld, per, bits);
     } else if (axis == 0) {
         k_amax_channels_elementwise<WIDE, 0><<<grid_for(rows * cols), kThreads, 0, st>>>(x, rows, cols, ld, bits);
     } else {
@@ -1023,10 +1040,10 @@ static fp8_status launch_quantize_channels(const void* x, int64_t rows, int64_t 
     }
     if (vec && axis == 0 && cols >= EPI) {
         const int64_t full_cols = cols / EPI * EPI;
-        const int64_t col_blocks = (full_cols / EPI + kThreads - 1) / kThreads;
+        const int64_t col_blocks = (full_cols / EPI + kColsTx - 1) / kColsTx;
         const int64_t per = slab_rows(rows, col_blocks);
         dim3 grid((unsigned)col_blocks, (unsigned)((rows + per - 1) / per));
-        k_quantize_cols<WIDE, FMT, NOSAT><<<grid, kThreads, 0, st>>>(x, rows, full_cols, ld, per, scale, out, ld_out);
+        k_quantize_cols<WIDE, FMT, NOSAT><<<grid, dim3(kColsTx, kColsTy), 0, st>>>(x, rows, full_cols, ld, per, scale, out, ld_out);
         count_launches(1);
         if (full_cols < cols) {
             k_quantize_channels_elementwise<WIDE, FMT, NOSAT, 0><<<grid_for(rows * (cols - full_cols)), kThreads, 0, st>>>(
