@@ -195,7 +195,7 @@ class LinearStep:
         events.append(row)
 
 
-def bench_cast_sweep(torch, api, synth, device, log2n, iters=5):
+def bench_cast_sweep(torch, api, synth, device, log2n, iters=20):
     """config-2 style bandwidth point: bf16 tensor of 2^log2n elements; single-pass quantize+amax, amax, dequantize"""
     n = 1 << log2n
     x = synth.normal_laplace_mixture(n, 1, synth.T_ID, device=device)
@@ -212,17 +212,21 @@ def bench_cast_sweep(torch, api, synth, device, log2n, iters=5):
         "amax": (lambda: api.fp8_amax(x, a), 2.0 * n),
         "quantize_current_e4m3": (lambda: api.fp8_quantize_current(x, api.E4M3, codes, a, s2, si2), 5.0 * n),
         "dequantize_e4m3": (lambda: api.fp8_dequantize(codes, api.E4M3, si, back), 3.0 * n),
+        "fake_quantize_e4m3": (lambda: api.fp8_fake_quantize(x, api.E4M3, s, si, back), 4.0 * n),
     }
     for name, (fn, nbytes) in cases.items():
         for _ in range(3):
             fn()
-        times = []
+        torch.cuda.synchronize()
+        # `iters` calls back to back between two events: the tensor (0.5 GB at 2^28) is far larger than L2,
+        # and launch gaps overlap with the previous call's tail as they do inside a real step
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         for _ in range(iters):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(); fn(); e1.record()
-            torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1))
-        ms = statistics.median(times)
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
         out[name] = {"ms": round(ms, 4), "gbs": round(nbytes / ms / 1e6, 1)}
     del x, codes, back
     torch.cuda.empty_cache()
