@@ -411,6 +411,10 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.next_rows_only:
+        # profiling aid: only the kernels beyond the core path, each on workload-shaped tensors
+        print(json.dumps({"next_rows": bench_next_rows(torch, api, synth, device, peaks(), iters=max(1, min(args.steps, 5)))}))
+        return
     # independent batches per rank: no data-path collective (per-tensor amax is local to a rank's own tensors)
     step = LinearStep(torch, api, synth, device, seed=3 + 16 * rank, fused_cast=not args.unfused_cast)
     if args.only:
@@ -568,6 +572,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cast-sweep", action="store_true")
     ap.add_argument("--no-next-rows", action="store_true")
+    ap.add_argument("--next-rows-only", action="store_true", help="profiling aid: run only the next-row kernels")
     ap.add_argument("--cast-log2n", type=int, default=28)
     ap.add_argument("--unfused-cast", action="store_true", help="amax, scale and quantize as three calls per tensor instead of fp8_quantize_current")
     ap.add_argument("--only", default=None, help="profiling aid: time only the calls with this label (e.g. gemm_fprop, quantize, amax)")
