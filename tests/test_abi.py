@@ -62,3 +62,40 @@ def test_argument_errors_are_reported_before_any_launch():
     assert lib.fp8_gemm(ctypes.byref(d), ctypes.c_void_p(24), one, one, one, one, None, None) == 4
     d.ldd = 100                                                                         # smaller than N
     assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 3
+
+
+def test_argument_errors_of_the_wider_entry_points():
+    lib = api.load()
+    one = ctypes.c_void_p(16)
+    # one-launch current scaling: null pointers, enums, workspace alignment
+    assert lib.fp8_quantize_current(one, 1, 4, 0, 0, one, None, one, one, one, None) == 1
+    assert lib.fp8_quantize_current(one, 1, 4, 0, 0, one, one, one, one, None, None) == 1
+    assert lib.fp8_quantize_current(one, 1, 4, 5, 0, one, one, one, one, one, None) == 2
+    assert lib.fp8_quantize_current(one, 1, 4, 0, 0, one, one, one, one, ctypes.c_void_p(24), None) == 4
+    assert lib.fp8_quantize_current_workspace_bytes() == 16
+    assert lib.fp8_quantize_current_static(one, 1, 4, 0, 0, one, None, one, one, None) == 1
+    assert lib.fp8_quantize_current_static(one, 9, 4, 0, 0, one, one, one, one, None) == 2
+    # simulated FP8, power-of-two scale
+    assert lib.fp8_fake_quantize(one, 1, 4, 0, 0, None, one, one, None) == 1
+    assert lib.fp8_fake_quantize(one, 1, 4, 0, 7, one, one, one, None) == 2
+    assert lib.fp8_scale_pow2_from_amax(one, 0, None, one, None) == 1
+    assert lib.fp8_scale_pow2_from_amax(one, 3, one, one, None) == 2
+    # per-channel
+    assert lib.fp8_amax_channels(one, 1, 4, 4, 4, 0, None, None) == 1
+    assert lib.fp8_amax_channels(one, 1, 4, 4, 4, 2, one, None) == 2
+    assert lib.fp8_amax_channels(one, 1, 4, 8, 4, 0, one, None) == 3            # pitch smaller than the row
+    assert lib.fp8_scales_from_amax(None, 4, 0, 0, one, one, None) == 1
+    assert lib.fp8_scales_from_amax(one, -1, 0, 0, one, one, None) == 3
+    assert lib.fp8_quantize_channels(one, 1, 4, 4, 4, 0, 0, 0, None, one, 4, None) == 1
+    assert lib.fp8_quantize_channels(one, 1, 4, 4, 4, 0, 0, 0, one, one, 2, None) == 3
+    assert lib.fp8_quantize_channels(one, 1, 4, 4, 4, 1, 4, 0, one, one, 4, None) == 2
+    # GEMM variants
+    d = api.GemmDesc(256, 256, 128, 0, 0, 0, 0, 128, 128, 256, 1)
+    assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 0, 0, one, one, None, None, None) == 1
+    assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 2, 0, one, one, one, None, None) == 2
+    assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 0, 3, one, one, one, None, None) == 2
+    assert lib.fp8_gemm_channel_scales(ctypes.byref(d), one, one, one, one, None, None, None) == 1
+    assert lib.fp8_gemm_batched(ctypes.byref(d), -1, one, 0, one, 0, one, 0, one, one, None, None) == 3
+    assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 100, one, 256 * 128, one, 256 * 256, one, one, None, None) == 3   # members overlap
+    assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 256 * 128 + 8, one, 256 * 128, one, 256 * 256, one, one, None, None) == 4
+    assert lib.fp8_gemm_batched(ctypes.byref(d), 70000, one, 256 * 128, one, 256 * 128, one, 256 * 256, one, one, None, None) == 5
