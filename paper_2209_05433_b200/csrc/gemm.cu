@@ -516,11 +516,17 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     if (lane == 0) bulk_wait_read<1>();           // the box stored two chunks ago has left this buffer
                     __syncwarp();
                 }
+                // TMEM loads go out two at a time (one wait for both) where a box spans several loads
+                constexpr int PRE = SUBS >= 2 ? 2 : 1;
+                uint32_t rr[PRE][32];
 #pragma unroll
                 for (int sub = 0; sub < SUBS; ++sub) {
-                    uint32_t r[32];
-                    tc_ld32(taddr + c * CHUNK + sub * 32, r);
-                    tc_wait_ld();
+                    if (sub % PRE == 0) {
+#pragma unroll
+                        for (int g = 0; g < PRE; ++g) tc_ld32(taddr + c * CHUNK + (sub + g) * 32, rr[g]);
+                        tc_wait_ld();
+                    }
+                    uint32_t (&r)[32] = rr[sub % PRE];
                     float v[32];
                     if (p.sb_inv_vec) {                       // per-channel weight scales: one alpha per column
                         const int64_t scol_v = col + sub * 32;
