@@ -62,8 +62,10 @@ constexpr int BK = 128;             // K-block in elements = bytes = one 128B sw
 constexpr int UMMA_K = 32;          // K of one tcgen05.mma for 8-bit operands
 constexpr int MAX_STAGES = 6;
 constexpr int ACC_STAGES = 2;       // 2 x 256 columns = all 512 TMEM columns
-constexpr int THREADS = 192;
-constexpr int EPI_WARPS = 4;
+// Epilogue width: 4 warps with two staging buffers each (long K: the epilogue has slack, fewer resident warps
+// leave the MMA-issuing thread undisturbed) or 8 warps with one buffer each (short K: the kernel is bound by
+// its output stream; two warps per TMEM lane quarter split the tile's columns).
+constexpr int SHORT_K_BLOCKS = 8;   // K <= 1024: eight epilogue warps
 constexpr uint32_t A_BYTES = BM * BK;          // 16 KiB: this CTA's 128 rows of A
 // per CTA group size: B bytes staged by one CTA, stage size, ring depth (192 KiB of tiles either way)
 template <int CG> struct Geo {
@@ -75,7 +77,7 @@ template <int CG> struct Geo {
 };
 constexpr uint32_t SMEM_TILES = 4 * (A_BYTES + BN * BK);            // = 6 * (A_BYTES + BN/2 * BK)
 constexpr uint32_t EPI_BUF_BYTES = 4096;                            // 32 rows x 128 B, one TMA store box
-constexpr uint32_t SMEM_EPI = EPI_WARPS * 2 * EPI_BUF_BYTES;        // two staging buffers per epilogue warp
+constexpr uint32_t SMEM_EPI = 8 * EPI_BUF_BYTES;                    // staging buffers of the epilogue warps (4 x 2 or 8 x 1)
 constexpr uint32_t SMEM_BARRIERS = 256;
 constexpr uint32_t SMEM_BYTES = SMEM_TILES + SMEM_EPI + SMEM_BARRIERS + 1024;   // + slack to align the ring to 1024 B
 constexpr uint32_t TMEM_COLS = 512;
@@ -317,11 +319,12 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 // CG: CTAs per tile (1 or 2).  OUT: what the epilogue writes (fp32, bf16, E4M3 or E5M2 codes).
 // Operand layouts (K-major or MN-major) are run-time properties: they only change TMA coordinates and
 // shared-memory descriptor constants.
-template <int CG, int OUT>
-__global__ void __launch_bounds__(THREADS, 1)
+template <int CG, int OUT, int EPI_WARPS>
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
            const __grid_constant__ CUtensorMap map_d, const Params p) {
     using G = Geo<CG>;
+    constexpr int EPI_BUFS = 8 / EPI_WARPS;
     constexpr int STAGES = G::STAGES;
     constexpr uint32_t STAGE_BYTES = G::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
@@ -480,7 +483,9 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         const float alpha = p.sb_inv_vec ? 0.0f : sa_inv * __ldg(p.sb_inv);
         const float scale_d = (OUT == OUT_E4M3 || OUT == OUT_E5M2) ? __ldg(p.scale_d) : 1.0f;
         uint32_t running = 0;                                     // max of stored magnitude bits (bf16: 16-bit patterns)
-        const uint32_t epi_base = ring + SMEM_TILES + (uint32_t)(warp - 2) * 2u * EPI_BUF_BYTES;
+        const uint32_t epi_base = ring + SMEM_TILES + (uint32_t)(warp - 2) * (uint32_t)EPI_BUFS * EPI_BUF_BYTES;
+        constexpr int COL_SPLIT = EPI_WARPS / 4;                  // warps sharing a lane quarter split the columns
+        const int col_part = (warp - 2) >> 2;
         uint32_t buf = 0;
         const uint64_t stream_out = policy_evict_first();
         bool ok = true;
@@ -505,7 +510,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             constexpr int SUBS = CHUNK / 32;                      // 32-column TMEM loads per box
             constexpr int WORDS = 32 * ESZ / 4;                   // 32-bit words one load contributes to the row
 #pragma unroll 1
-            for (int c = 0; c < BN / CHUNK; ++c) {
+            for (int c = col_part * (BN / CHUNK / COL_SPLIT); c < (col_part + 1) * (BN / CHUNK / COL_SPLIT); ++c) {
                 const int64_t col = col0 + (int64_t)c * CHUNK;
                 // A box that crosses the right edge is clipped by the TMA unit in 16-byte units: when the row
                 // length in bytes is not a multiple of 16 that last box is written with plain stores instead.
@@ -513,7 +518,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 const uint32_t sbuf = epi_base + buf * EPI_BUF_BYTES;
                 const uint32_t srow = sbuf + lane * 128;
                 if (!direct) {
-                    if (lane == 0) bulk_wait_read<1>();           // the box stored two chunks ago has left this buffer
+                    if (lane == 0) bulk_wait_read<EPI_BUFS - 1>();  // the box last stored from this buffer has left it
                     __syncwarp();
                 }
                 // TMEM loads go out two at a time (one wait for both) where a box spans several loads
@@ -597,7 +602,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     if (row0 < p.M && col < p.N) tma_store_3d(&map_d, sbuf, (int)(col * ESZ), row0, bi, stream_out);
                     bulk_commit();
                 }
-                buf ^= 1u;
+                buf = (buf + 1u) % (uint32_t)EPI_BUFS;
             }
             tc_fence_before();
             __syncwarp();
@@ -660,9 +665,10 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
 }
 
 // CTA-pair kernels launch as clusters of 2; the grid is one CTA per SM that can be paired.
-template <int CG, int OUT>
+template <int CG, int OUT, int EPI_WARPS>
 static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const Params& p, int64_t num_tiles, cudaStream_t st) {
-    auto k = k_gemm_fp8<CG, OUT>;
+    auto k = k_gemm_fp8<CG, OUT, EPI_WARPS>;
+    constexpr int THREADS = 64 + 32 * EPI_WARPS;
     // per device and cheap, so set on every launch rather than cached
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return FP8_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -691,13 +697,21 @@ static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
 }
 
 template <int CG>
-static fp8_status dispatch(int out_kind, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
+static fp8_status dispatch(int out_kind, bool short_k, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
                            const Params& p, int64_t num_tiles, cudaStream_t st) {
+    if (short_k) {
+        switch (out_kind) {
+            case OUT_F32:  return launch<CG, OUT_F32, 8>(ma, mb, md, p, num_tiles, st);
+            case OUT_BF16: return launch<CG, OUT_BF16, 8>(ma, mb, md, p, num_tiles, st);
+            case OUT_E4M3: return launch<CG, OUT_E4M3, 8>(ma, mb, md, p, num_tiles, st);
+            default:       return launch<CG, OUT_E5M2, 8>(ma, mb, md, p, num_tiles, st);
+        }
+    }
     switch (out_kind) {
-        case OUT_F32:  return launch<CG, OUT_F32>(ma, mb, md, p, num_tiles, st);
-        case OUT_BF16: return launch<CG, OUT_BF16>(ma, mb, md, p, num_tiles, st);
-        case OUT_E4M3: return launch<CG, OUT_E4M3>(ma, mb, md, p, num_tiles, st);
-        default:       return launch<CG, OUT_E5M2>(ma, mb, md, p, num_tiles, st);
+        case OUT_F32:  return launch<CG, OUT_F32, 4>(ma, mb, md, p, num_tiles, st);
+        case OUT_BF16: return launch<CG, OUT_BF16, 4>(ma, mb, md, p, num_tiles, st);
+        case OUT_E4M3: return launch<CG, OUT_E4M3, 4>(ma, mb, md, p, num_tiles, st);
+        default:       return launch<CG, OUT_E5M2, 4>(ma, mb, md, p, num_tiles, st);
     }
 }
 
@@ -774,8 +788,9 @@ static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint
     // instruction descriptor: fp32 accumulate, operand formats and majors, N/8, M/16 (M = 256 for a CTA pair)
     p.idesc = (1u << 4) | ((uint32_t)d->fa << 7) | ((uint32_t)d->fb << 10) | ((a_mn ? 1u : 0u) << 15) |
               ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
-    return cg == 2 ? dispatch<2>(out_kind, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st)
-                   : dispatch<1>(out_kind, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st);
+    const bool short_k = (K + BK - 1) / BK <= SHORT_K_BLOCKS;
+    return cg == 2 ? dispatch<2>(out_kind, short_k, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st)
+                   : dispatch<1>(out_kind, short_k, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st);
 }
 
 }  // namespace gemm
