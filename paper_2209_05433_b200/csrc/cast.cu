@@ -933,7 +933,10 @@ static fp8_status launch_current(const void* x, size_t n, float fmax, uint8_t* o
     if (chunks < 1) chunks = 1;
     const int grid = persistent_grid(k, chunks);               // co-resident by construction: SMs x occupancy at most
     void* args[] = {(void*)&x, (void*)&n, (void*)&fmax, (void*)&out, (void*)&amax, (void*)&scale, (void*)&scale_inv, (void*)&ws};
-    if (cudaLaunchCooperativeKernel((const void*)k, dim3(grid), dim3(kThreads), args, 0, st) != cudaSuccess) return FP8_ERR_CUDA;
+    if (cudaLaunchCooperativeKernel((const void*)k, dim3(grid), dim3(kThreads), args, 0, st) != cudaSuccess) {
+        (void)cudaGetLastError();                                  // e.g. the device cannot hold the whole grid right now
+        return FP8_ERR_UNSUPPORTED;                                // the caller falls back to the three separate kernels
+    }
     count_launches(1);
     return launch_status();
 }
@@ -951,16 +954,24 @@ fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_form
     }
     const float fmax = f == FP8_E4M3 ? 448.0f : 57344.0f;
     const bool nosat = o == FP8_NOSAT;
+    fp8_status s;
     if (t == FP8_F32) {
-        if (f == FP8_E4M3) return nosat ? launch_current<kWideF32, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
-                                        : launch_current<kWideF32, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
-        return nosat ? launch_current<kWideF32, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
-                     : launch_current<kWideF32, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+        if (f == FP8_E4M3) s = nosat ? launch_current<kWideF32, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                     : launch_current<kWideF32, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+        else               s = nosat ? launch_current<kWideF32, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                     : launch_current<kWideF32, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+    } else {
+        if (f == FP8_E4M3) s = nosat ? launch_current<kWideBF16, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                     : launch_current<kWideBF16, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+        else               s = nosat ? launch_current<kWideBF16, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                     : launch_current<kWideBF16, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
     }
-    if (f == FP8_E4M3) return nosat ? launch_current<kWideBF16, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
-                                    : launch_current<kWideBF16, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
-    return nosat ? launch_current<kWideBF16, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
-                 : launch_current<kWideBF16, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+    if (s == FP8_ERR_UNSUPPORTED) {                                // cooperative launch refused: same results, three launches
+        s = fp8_amax(x, t, n, amax, st);
+        if (s == FP8_OK) s = fp8_scale_from_amax(amax, f, scale, scale_inv, st);
+        if (s == FP8_OK) s = fp8_quantize(x, t, n, f, o, scale, out, nullptr, st);
+    }
+    return s;
 }
 
 template <int WIDE, int FMT, bool NOSAT>

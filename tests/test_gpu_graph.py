@@ -1,0 +1,66 @@
+"""The whole linear-layer step (casts + three GEMMs) captured once in a CUDA graph and replayed:
+the library makes no host synchronisation, allocation or host-side read of device scalars on the way,
+and a replay on new input values gives exactly what eager calls give."""
+import pytest
+import torch
+
+from paper_2209_05433_b200 import api, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _step(X, W, dY, buf, fused):
+    T, I = X.shape
+    O = W.shape[1]
+    s = buf["scal"]
+    ax, sx, six, aw, sw, siw, ag, sg, sig, ay, adx, adw = [s[i:i + 1] for i in range(12)]
+    if fused:
+        api.fp8_quantize_current(X, api.E4M3, buf["Xq"], ax, sx, six)
+        api.fp8_quantize_current(W, api.E4M3, buf["Wq"], aw, sw, siw)
+        api.fp8_quantize_current(dY, api.E5M2, buf["Gq"], ag, sg, sig)
+    else:
+        for t, q, fmt, a, sc, si in ((X, buf["Xq"], api.E4M3, ax, sx, six), (W, buf["Wq"], api.E4M3, aw, sw, siw),
+                                     (dY, buf["Gq"], api.E5M2, ag, sg, sig)):
+            api.fp8_amax(t, a)
+            api.fp8_scale_from_amax(a, fmt, sc, si)
+            api.fp8_quantize(t, fmt, sc, q)
+    api.fp8_gemm(buf["Xq"], api.E4M3, api.MAJOR_K, buf["Wq"], api.E4M3, api.MAJOR_MN, buf["Y"], six, siw, ay)
+    api.fp8_gemm(buf["Gq"], api.E5M2, api.MAJOR_K, buf["Wq"], api.E4M3, api.MAJOR_K, buf["dX"], sig, siw, adx)
+    api.fp8_gemm(buf["Xq"], api.E4M3, api.MAJOR_MN, buf["Gq"], api.E5M2, api.MAJOR_MN, buf["dW"], six, sig, adw)
+
+
+def _buffers(T, I, O):
+    u8, bf = torch.uint8, torch.bfloat16
+    return {"Xq": torch.empty(T, I, dtype=u8, device=DEV), "Wq": torch.empty(I, O, dtype=u8, device=DEV),
+            "Gq": torch.empty(T, O, dtype=u8, device=DEV), "Y": torch.empty(T, O, dtype=bf, device=DEV),
+            "dX": torch.empty(T, I, dtype=bf, device=DEV), "dW": torch.empty(I, O, dtype=bf, device=DEV),
+            "scal": torch.zeros(16, dtype=torch.float32, device=DEV)}
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_step_replays_from_a_cuda_graph(fused):
+    T, I, O = 512, 384, 768
+    X = synth.activations(T * I, 3, device=DEV).view(T, I)
+    W = synth.weights(I * O, 3, 0.02, device=DEV).view(I, O)
+    dY = synth.gradients(T * O, 4, device=DEV).view(T, O)
+    graph_buf, eager_buf = _buffers(T, I, O), _buffers(T, I, O)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        api.current_scaling_workspace(X.device)            # the workspace of this stream exists before the capture
+        _step(X, W, dY, graph_buf, fused)                   # warm-up outside the capture (first-use set-up)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            _step(X, W, dY, graph_buf, fused)
+    torch.cuda.synchronize()
+    for trial in range(2):
+        # new values in the same input buffers, then replay
+        X.copy_(synth.activations(T * I, 30 + trial, device=DEV).view(T, I))
+        dY.copy_(synth.gradients(T * O, 40 + trial, device=DEV).view(T, O) * (3.0 + trial))
+        g.replay()
+        _step(X, W, dY, eager_buf, fused)
+        torch.cuda.synchronize()
+        assert api.fp8_async_status()[0] == 0
+        for k in graph_buf:
+            assert torch.equal(graph_buf[k].view(torch.uint8), eager_buf[k].view(torch.uint8)), (k, trial)
