@@ -233,6 +233,33 @@ def bench_cast_sweep(torch, api, synth, device, log2n, iters=20):
     return out
 
 
+def bench_gemm_alone(torch, step, seconds=2.0):
+    """The forward GEMM of the step by itself: best single launch (burst) and a back-to-back loop of at
+    least `seconds` (sustained, under the power cap)."""
+    call = dict(step.calls())["gemm_fprop"]
+    flops = 2.0 * step.T * step.I * step.O
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    best = 1e9
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); call(); e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    n = max(10, int(seconds * 1e3 / best))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    return {"shape": "M=%d N=%d K=%d, E4M3 x E4M3 -> bf16" % (step.T, step.O, step.I),
+            "burst_tflops": round(flops / best / 1e9, 1), "sustained_tflops": round(flops / ms / 1e9, 1),
+            "sustained_launches": n, "sustained_seconds": round(ms * n / 1e3, 2)}
+
+
 def bench_next_rows(torch, api, synth, device, pk, iters=5):
     """The rows beyond the core path, each timed alone on workload-shaped tensors: simulated-FP8 round trip,
     per-channel weight scales, FP8-output GEMM, attention-style batched GEMM."""
@@ -560,6 +587,7 @@ def run_ours(args):
             cast = bench_cast_sweep(torch, api, synth, device, args.cast_log2n)
             for v in cast.values():
                 v["frac_of_measured_hbm"] = round(v["gbs"] / pk["hbm_gbs"], 4)
+        gemm_alone = bench_gemm_alone(torch, step) if world == 1 and not args.no_next_rows else None
         next_rows = None
         if world == 1 and not args.no_next_rows:
             next_rows = bench_next_rows(torch, api, synth, device, pk)
@@ -581,6 +609,7 @@ def run_ours(args):
                     "how": "pinned host buffers; upload, kernels and download of consecutive steps overlap on three streams"},
             "gpu_launches": int(launches), "gpu_launches_note": "kernels plus 4-byte memset nodes enqueued by the library in the timed region",
             "roofline": roofline, "roofline_cast": roofline_cast, "kernels": kernels, "cast_sweep_2pow%d" % args.cast_log2n: cast,
+            "gemm_alone": gemm_alone,
             "next_rows": next_rows,
             "cpu_baseline": cpu,
         }

@@ -63,6 +63,8 @@ def _load():
     lib.fp8o_f64_to_bf16.argtypes = [c.c_double]
     lib.fp8o_f64_to_bf16_array.restype = None
     lib.fp8o_f64_to_bf16_array.argtypes = [f64p, c.c_size_t, u16p]
+    lib.fp8o_count_double_rounding_f32.restype = c.c_size_t
+    lib.fp8o_count_double_rounding_f32.argtypes = [f32p, c.c_size_t, c.c_float, c.c_int, c.c_int]
     lib.fp8o_quantize_f32.restype = None
     lib.fp8o_quantize_f32.argtypes = [f32p, c.c_size_t, c.c_float, c.c_int, c.c_int, u8p]
     lib.fp8o_quantize_bf16.restype = None
@@ -194,6 +196,13 @@ def quantize(x: np.ndarray, scale, fmt: int, overflow: int = SATURATE, threads: 
                 _ptr(x[lo:hi], ctypes.c_uint16), hi - lo, sc, fmt, overflow, _ptr(out[lo:hi], ctypes.c_uint8)))
     _run(jobs, threads)
     return out
+
+
+def count_double_rounding(x: np.ndarray, scale, fmt: int, overflow: int = SATURATE) -> int:
+    """Diagnostic: elements whose code would differ if the exact product x*scale were rounded once
+    (instead of to binary32 first, then to FP8)."""
+    x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
+    return int(_load().fp8o_count_double_rounding_f32(_ptr(x, ctypes.c_float), x.size, ctypes.c_float(np.float32(scale)), fmt, overflow))
 
 
 def dequantize(codes: np.ndarray, scale_inv, fmt: int, wide: str = "f32", threads: int = 1) -> np.ndarray:

@@ -179,6 +179,47 @@ uint8_t fp8o_encode(float y, int fmt, int overflow)
     return (uint8_t)((s << 7) | (uint32_t)mag);
 }
 
+/* Diagnostic for the reading "two roundings" of the scale multiply: the code a
+ * SINGLE rounding of the exact product x*scale would give.  The product of two
+ * binary32 values is exact in double, so this is the conversion of that double:
+ * same steps as fp8o_encode on a 53-bit significand. */
+uint8_t fp8o_encode_exact_product(float x, float scale, int fmt, int overflow)
+{
+    const int emin  = (fmt == FP8O_E4M3) ? -6 : -14;
+    const int mbits = (fmt == FP8O_E4M3) ? 3 : 2;
+    const int bias  = (fmt == FP8O_E4M3) ? 7 : 15;
+    const uint32_t maxmag = (fmt == FP8O_E4M3) ? 0x7Eu : 0x7Bu;
+    double y = (double)x * (double)scale;
+    uint32_t s = signbit(y) ? 1u : 0u;
+    if (isnan(y)) return (uint8_t)(((signbit(x) ? 1u : 0u) << 7) | 0x7Fu);
+    double a = fabs(y);
+    if (isinf(a) || a >= ldexp(1.0, 128) * (1.0 - ldexp(1.0, -25)))       /* rounds to binary32 infinity */
+        return (uint8_t)((s << 7) | (fmt == FP8O_E4M3 ? 0x7Fu : 0x7Cu));
+    if (a == 0.0) return (uint8_t)(s << 7);
+    int e;
+    (void)frexp(a, &e);
+    int q = e - 1;
+    if (q < emin) q = emin;
+    double t = ldexp(a, -(q - mbits));                 /* |y| in units of the rounding quantum, exact */
+    double k = floor(t), rem = t - k;
+    if (rem > 0.5 || (rem == 0.5 && fmod(k, 2.0) == 1.0)) k += 1.0;
+    uint64_t ki = (uint64_t)k, mag;
+    if (q == emin) mag = ki;
+    else mag = ((uint64_t)(q + bias) << mbits) + (ki - ((uint64_t)1 << mbits));
+    if (mag > maxmag) mag = (overflow == FP8O_SATURATE) ? maxmag : (fmt == FP8O_E4M3 ? 0x7Fu : 0x7Cu);
+    return (uint8_t)((s << 7) | (uint32_t)mag);
+}
+
+/* how many elements would get a different code under the single-rounding reading */
+size_t fp8o_count_double_rounding_f32(const float* x, size_t n, float scale, int fmt, int overflow)
+{
+    size_t c = 0;
+    for (size_t i = 0; i < n; ++i)
+        c += fp8o_encode_exact_product(x[i], scale, fmt, overflow) != fp8o_encode((float)((double)x[i] * (double)scale), fmt, overflow)
+             && !isnan(x[i]);
+    return c;
+}
+
 /* ------------------------------------------------------ quantize / dequantize */
 
 /* one IEEE binary32 multiply: the double product of two floats is exact

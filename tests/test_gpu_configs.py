@@ -44,7 +44,7 @@ def _cast(x, fmt, rng):
     return codes, si, codes_host, wsi
 
 
-def _sample_positions(M, N, rng, n_random=4096, n_tiles=64):
+def _sample_positions(M, N, rng, n_random=16384, n_tiles=64):
     ii = [np.zeros(N, dtype=np.int64), np.full(N, M - 1, dtype=np.int64)]
     jj = [np.arange(N, dtype=np.int64), np.arange(N, dtype=np.int64)]
     tm = rng.integers(0, (M + 127) // 128, size=n_tiles)

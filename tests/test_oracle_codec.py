@@ -337,6 +337,24 @@ def test_round_trip_error_bound(fmt, mbits):
     assert np.all(np.abs(xh[small].astype(np.float64) - x[small]) <= quantum / 2 * (1 + 1e-5))
 
 
+def test_double_rounding_diagnostic():
+    # two roundings (binary32 product, then FP8) against one rounding of the exact product: they can only
+    # differ when the binary32 rounding lands on an FP8 tie, which is rare but real
+    rng = np.random.default_rng(33)
+    x = rng.standard_normal(1 << 20).astype(np.float32)
+    for fmt in (E4M3, E5M2):
+        n = oracle.count_double_rounding(x, np.float32(37.123), fmt)
+        assert 0 <= n < x.size // 10000
+        assert oracle.count_double_rounding(x, np.float32(2.0), fmt) == 0        # a power-of-two scale multiplies exactly
+    # a constructed case: x*scale exactly just above the E4M3 tie 1.0625, its binary32 rounding exactly on the tie
+    xs = np.array([np.float32(1.0625) + np.float32(2.0 ** -23)], dtype=np.float32)   # 1.0625 + 1 ulp
+    sc = np.float32(1.0 - 2.0 ** -24)                                                 # product = 1.0625 + ~2^-23 - 2^-24*1.0625...
+    exact = float(xs[0]) * float(sc)
+    assert exact > 1.0625 and np.float32(exact) == np.float32(1.0625)
+    assert oracle.count_double_rounding(xs, sc, E4M3) == 1                            # exact -> 0x39, twice rounded -> tie -> 0x38
+    assert oracle.quantize(xs, sc, E4M3)[0] == 0x38
+
+
 # ------------------------------------------------------------ amax / scale --
 
 def test_amax_closed_form_and_nan():
