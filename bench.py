@@ -308,6 +308,16 @@ def bench_next_rows(torch, api, synth, device, pk, iters=5):
     out["gemm_fprop_channel_scales"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
     ms = timed(lambda: api.fp8_gemm_fp8out(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Yq, api.E4M3, sx[2:3], si, s, a))
     out["gemm_fprop_fp8_output"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
+    # split accumulation (partial sums every 2048 of K added in registers): forward K = 4096 and, on the same codes
+    # read as dY-shaped operands, the dgrad shape K = 16384
+    ms = timed(lambda: api.fp8_gemm(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, sx[2:3], si, a, acc=api.ACC_SPLIT))
+    out["gemm_fprop_split_accumulation"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
+    dX = torch.empty(TOKENS, D_IN, dtype=torch.bfloat16, device=device)
+    ms = timed(lambda: api.fp8_gemm(Yq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, si, si, a, acc=api.ACC_SPLIT))
+    out["gemm_dgrad_split_accumulation"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
+    ms = timed(lambda: api.fp8_gemm(Yq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, si, si, a))
+    out["gemm_dgrad_same_codes_one_accumulator"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
+    del dX
     del W, X, Y, Yq
     # attention-style batched products: 32 heads, 4096 tokens, head dim 128: scores = Q.K^T, context = P.V
     H, S, Dh = 32, 4096, 128

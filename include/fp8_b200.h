@@ -48,6 +48,8 @@ typedef enum { FP8_F32 = 0, FP8_BF16 = 1 } fp8_wide;
 typedef enum { FP8_SATURATE = 0, FP8_NOSAT = 1 } fp8_overflow;
 /* Which index of a GEMM operand is contiguous in memory. */
 typedef enum { FP8_MAJOR_K = 0, FP8_MAJOR_MN = 1 } fp8_major;
+/* how a GEMM accumulates over K (see fp8_gemm) */
+typedef enum { FP8_ACC_FAST = 0, FP8_ACC_SPLIT = 1 } fp8_accumulate;
 
 /*
  * fp8_amax — maximum magnitude of a tensor (Section 2: the quantity the scale
@@ -193,6 +195,15 @@ fp8_status fp8_scale_pow2_from_amax(const float* amax_dev, fp8_format f,
  * be multiples of 16, else FP8_ERR_ALIGN.  M, N, K are otherwise arbitrary
  * (edges are zero-filled on load and clipped on store).  M*N == 0 is a no-op
  * (amax = 0); K == 0 writes zeros.
+ * Accumulation (`acc`): the products are exact and the tensor core adds them, 32 of K at a time, into a
+ * binary32 accumulator whose additions round toward zero.
+ *   FP8_ACC_FAST   one accumulator over all of K.  The error is below 1e-5 * sum_k|a.b| for K <= 2048 on any
+ *                  data, and for any K when the products are mixed in sign (training tensors); products of
+ *                  one sign lose up to (K/32) * 2^-23 of their sum.
+ *   FP8_ACC_SPLIT  the accumulator is drained every 2048 of K and the partial sums are added in registers
+ *                  with round-to-nearest: below 1e-5 * sum_k|a.b| for any data and any K, at a cost of a few
+ *                  per cent of throughput.  Identical to FAST for K <= 2048.
+ * Every GEMM entry point that takes this descriptor honours `acc`; other values give FP8_ERR_ENUM.
  */
 typedef struct {
     int64_t M, N, K;
@@ -200,6 +211,7 @@ typedef struct {
     fp8_major ma, mb;
     int64_t lda, ldb, ldd;
     fp8_wide out;
+    fp8_accumulate acc;
 } fp8_gemm_desc;
 
 fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,

@@ -18,6 +18,7 @@ E4M3, E5M2 = 0, 1            # fp8_format
 F32, BF16 = 0, 1             # fp8_wide
 SATURATE, NOSAT = 0, 1       # fp8_overflow
 MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
+ACC_FAST, ACC_SPLIT = 0, 1    # fp8_accumulate
 
 EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
            "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_fake_quantize",
@@ -33,7 +34,7 @@ class Fp8Error(RuntimeError):
 class GemmDesc(ctypes.Structure):
     _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
                 ("fa", ctypes.c_int), ("fb", ctypes.c_int), ("ma", ctypes.c_int), ("mb", ctypes.c_int),
-                ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldd", ctypes.c_int64), ("out", ctypes.c_int)]
+                ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldd", ctypes.c_int64), ("out", ctypes.c_int), ("acc", ctypes.c_int)]
 
 
 _lib = None
@@ -212,12 +213,15 @@ def fp8_scale_pow2_from_amax(amax: torch.Tensor, fmt: int, scale_out: torch.Tens
 
 
 def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
-             scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, amax_out: torch.Tensor | None = None) -> None:
+             scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, amax_out: torch.Tensor | None = None,
+             acc: int = ACC_FAST) -> None:
     """D[M,N] = (A[M,K] . B[K,N]) * scale_inv_a * scale_inv_b.
 
     A is a 2-D uint8 tensor stored [M,K] when ``ma == MAJOR_K`` or [K,M] when
     ``ma == MAJOR_MN``; B is stored [N,K] when ``mb == MAJOR_K`` or [K,N] when
-    ``mb == MAJOR_MN``.  Row pitches are taken from the tensors' strides."""
+    ``mb == MAJOR_MN``.  Row pitches are taken from the tensors' strides.
+    ``acc`` selects one accumulator over all of K (ACC_FAST) or partial sums every 2048 of K added in
+    registers (ACC_SPLIT: tolerance met on same-sign data at any K)."""
     if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
         raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D tensor")
     for t, name in ((A, "A"), (B, "B"), (D, "D")):
@@ -227,7 +231,7 @@ def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: in
     Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
     if K != Kb or tuple(D.shape) != (M, N):
         raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
-    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D))
+    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D), acc)
     _check(load().fp8_gemm(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
                            _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
                            None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()), "fp8_gemm")
@@ -235,7 +239,7 @@ def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: in
 
 def fp8_gemm_fp8out(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor, fd: int,
                     scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, scale_d: torch.Tensor,
-                    amax_out: torch.Tensor | None = None, overflow: int = SATURATE) -> None:
+                    amax_out: torch.Tensor | None = None, overflow: int = SATURATE, acc: int = ACC_FAST) -> None:
     """D[M,N] (uint8 codes of format fd) = encode((A . B) * scale_inv_a * scale_inv_b * scale_d); amax_out
     receives the amax of the result before the output scale and conversion.  Layout rules as fp8_gemm."""
     if A.dtype != torch.uint8 or B.dtype != torch.uint8 or D.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
@@ -247,7 +251,7 @@ def fp8_gemm_fp8out(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int,
     Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
     if K != Kb or tuple(D.shape) != (M, N):
         raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
-    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), BF16)
+    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), BF16, acc)
     _check(load().fp8_gemm_fp8out(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(), fd, overflow,
                                   _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
                                   _scalar(scale_d, "scale_d"), None if amax_out is None else _scalar(amax_out, "amax_out"),
@@ -289,7 +293,8 @@ def fp8_quantize_channels(x: torch.Tensor, axis: int, fmt: int, scale_vec: torch
 
 
 def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
-                            scale_inv_a: torch.Tensor, scale_inv_b_vec: torch.Tensor, amax_out: torch.Tensor | None = None) -> None:
+                            scale_inv_a: torch.Tensor, scale_inv_b_vec: torch.Tensor, amax_out: torch.Tensor | None = None,
+                            acc: int = ACC_FAST) -> None:
     """fp8_gemm with one inverse scale per column of B (per output channel)."""
     if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
         raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D tensor")
@@ -300,7 +305,7 @@ def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, 
     Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
     if K != Kb or tuple(D.shape) != (M, N):
         raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
-    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D))
+    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D), acc)
     _check(load().fp8_gemm_channel_scales(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
                                           _scalar(scale_inv_a, "scale_inv_a"), _vec(scale_inv_b_vec, N, "scale_inv_b_vec"),
                                           None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()),
@@ -308,7 +313,8 @@ def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, 
 
 
 def fp8_gemm_batched(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
-                     scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, amax_out: torch.Tensor | None = None) -> None:
+                     scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, amax_out: torch.Tensor | None = None,
+                     acc: int = ACC_FAST) -> None:
     """Batched fp8_gemm: A, B are 3-D uint8 tensors [batch, rows, cols] (layouts per member as fp8_gemm), D is
     [batch, M, N]; the batch strides are taken from the tensors."""
     if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 3 or B.dim() != 3 or D.dim() != 3:
@@ -321,7 +327,7 @@ def fp8_gemm_batched(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int
     Kb, N = (B.shape[2], B.shape[1]) if mb == MAJOR_K else (B.shape[1], B.shape[2])
     if K != Kb or B.shape[0] != batch or tuple(D.shape) != (batch, M, N):
         raise ValueError("shape mismatch")
-    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(1), B.stride(1), D.stride(1), _wide_of(D))
+    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(1), B.stride(1), D.stride(1), _wide_of(D), acc)
     _check(load().fp8_gemm_batched(ctypes.byref(d), batch, A.data_ptr(), A.stride(0), B.data_ptr(), B.stride(0),
                                    D.data_ptr(), D.stride(0), _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
                                    None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()), "fp8_gemm_batched")

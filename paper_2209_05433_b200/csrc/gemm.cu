@@ -66,6 +66,7 @@ constexpr int ACC_STAGES = 2;       // 2 x 256 columns = all 512 TMEM columns
 // leave the MMA-issuing thread undisturbed) or 8 warps with one buffer each (short K: the kernel is bound by
 // its output stream; two warps per TMEM lane quarter split the tile's columns).
 constexpr int SHORT_K_BLOCKS = 8;   // K <= 1024: eight epilogue warps
+constexpr int SPLIT_BLOCKS = 16;    // split accumulation: the TMEM accumulator is drained into registers every 2048 of K
 constexpr uint32_t A_BYTES = BM * BK;          // 16 KiB: this CTA's 128 rows of A
 // per CTA group size: B bytes staged by one CTA, stage size, ring depth (192 KiB of tiles either way)
 template <int CG> struct Geo {
@@ -319,7 +320,11 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 // CG: CTAs per tile (1 or 2).  OUT: what the epilogue writes (fp32, bf16, E4M3 or E5M2 codes).
 // Operand layouts (K-major or MN-major) are run-time properties: they only change TMA coordinates and
 // shared-memory descriptor constants.
-template <int CG, int OUT, int EPI_WARPS>
+// SPLIT: split accumulation (needs 8 epilogue warps): the tensor core adds each K=32 block into the binary32
+// accumulator with truncation, so over a long K same-sign products lose up to (K/32) 2^-23 of their sum; here
+// the accumulator is closed every SPLIT_BLOCKS K-blocks and the partial sums are added in registers with
+// round-to-nearest, which keeps the error below 1e-5 of sum|a.b| for any data.
+template <int CG, int OUT, int EPI_WARPS, bool SPLIT>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
            const __grid_constant__ CUtensorMap map_d, const Params p) {
@@ -341,8 +346,10 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
     const int num_tiles = tiles_per_batch * p.batch;
     const int k_blocks = (int)((p.K + BK - 1) / BK);
     const bool A_MN = p.a_mn != 0, B_MN = p.b_mn != 0;
+    static_assert(!SPLIT || EPI_WARPS == 8, "split accumulation uses eight epilogue warps");
     constexpr int FG = G::FG;
     const int k_pad = (k_blocks + FG - 1) / FG * FG;               // K-blocks are consumed FG at a time
+    const int chunk_blocks = SPLIT ? SPLIT_BLOCKS : k_pad;         // K-blocks per use of a TMEM accumulator
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bars->full[s]), FG * CG); mbar_init(smem_u32(&bars->empty[s]), 1); }
@@ -427,7 +434,8 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         const uint32_t a_kstep = A_MN ? UMMA_K * 128 : UMMA_K, a_lbo = A_MN ? BK * 128 : 16;
         const uint32_t b_kstep = B_MN ? UMMA_K * 128 : UMMA_K, b_lbo = B_MN ? BK * 128 : 16;
         PROF_DECL
-        for (int t = worker; t < num_tiles && ok; t += num_workers, ++it) {
+        for (int t = worker; t < num_tiles && ok; t += num_workers) {
+          for (int kc = 0; kc < k_pad && ok; kc += chunk_blocks, ++it) {          // `it` counts accumulator uses
             const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
             PROF_BEGIN
             ok = mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag, WAIT_ACC_EMPTY);
@@ -435,7 +443,9 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             if (!ok) break;
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * BN;
-            for (int kb = 0; kb < k_pad; kb += FG) {
+            const int kend = min(k_pad, kc + chunk_blocks);
+            const int last_real = min(k_blocks, kend) - 1;                        // its MMAs complete the accumulator
+            for (int kb = kc; kb < kend; kb += FG) {
                 // one wait per TWO K-blocks: every barrier query between MMA issues costs about one MMA time
                 PROF_BEGIN
                 ok = mbar_wait(smem_u32(&bars->full[stage / FG]), phase, abort_flag, WAIT_FULL);
@@ -455,18 +465,18 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                                 // MN-major: 8-k groups 1024 B apart, 128-wide MN blocks BK*128 B apart, +32 k-rows per step.
                                 const uint64_t da = smem_desc(sa + k * a_kstep, a_lbo, 1024);
                                 const uint64_t db = smem_desc(sb + k * b_kstep, b_lbo, 1024);
-                                if (CG == 2) tc_mma_f8_pair(tmem_d, da, db, p.idesc, (kb | h | k) != 0 ? 1u : 0u);
-                                else         tc_mma_f8(tmem_d, da, db, p.idesc, (kb | h | k) != 0 ? 1u : 0u);
+                                if (CG == 2) tc_mma_f8_pair(tmem_d, da, db, p.idesc, ((kb - kc) | h | k) != 0 ? 1u : 0u);
+                                else         tc_mma_f8(tmem_d, da, db, p.idesc, ((kb - kc) | h | k) != 0 ? 1u : 0u);
                             }
                         }
                         // frees the smem stage (in both CTAs) when the MMAs retire (a padding block frees at once);
-                        // the last real block also publishes the accumulator
+                        // the last real block of the chunk also publishes the accumulator
                         if (CG == 2) {
                             tc_commit_pair(smem_u32(&bars->empty[st]));
-                            if (kb + h == k_blocks - 1) tc_commit_pair(smem_u32(&bars->acc_full[acc]));
+                            if (kb + h == last_real) tc_commit_pair(smem_u32(&bars->acc_full[acc]));
                         } else {
                             tc_commit(smem_u32(&bars->empty[st]));
-                            if (kb + h == k_blocks - 1) tc_commit(smem_u32(&bars->acc_full[acc]));
+                            if (kb + h == last_real) tc_commit(smem_u32(&bars->acc_full[acc]));
                         }
                     }
                 }
@@ -474,6 +484,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 stage += FG;
                 if (stage == STAGES) { stage = 0; phase ^= 1u; }
             }
+          }
         }
         PROF_STORE(3, 4, 5)
     } else {
@@ -491,10 +502,12 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         bool ok = true;
         int it = 0;
         PROF_DECL
-        for (int t = worker; t < num_tiles && ok; t += num_workers, ++it) {
-            int tm, tn;
-            const int bi = t / tiles_per_batch;
-            tile_coords(t - bi * tiles_per_batch, p.tiles_m, p.tiles_n, tm, tn);
+        float part[SPLIT ? 128 : 1];                              // split accumulation: this thread's 128 partial sums
+        for (int t = worker; t < num_tiles && ok; t += num_workers) {
+          int tm, tn;
+          const int bi = t / tiles_per_batch;
+          tile_coords(t - bi * tiles_per_batch, p.tiles_m, p.tiles_n, tm, tn);
+          for (int kc = 0; kc < k_pad && ok; kc += chunk_blocks, ++it) {         // `it` counts accumulator uses
             const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
             PROF_BEGIN
             ok = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, WAIT_ACC_FULL);
@@ -509,8 +522,31 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             constexpr int CHUNK = 128 / ESZ;                      // columns per staged box: 128 bytes per row
             constexpr int SUBS = CHUNK / 32;                      // 32-column TMEM loads per box
             constexpr int WORDS = 32 * ESZ / 4;                   // 32-bit words one load contributes to the row
-#pragma unroll 1
-            for (int c = col_part * (BN / CHUNK / COL_SPLIT); c < (col_part + 1) * (BN / CHUNK / COL_SPLIT); ++c) {
+            constexpr int NBOX = BN / CHUNK / COL_SPLIT;          // boxes per warp and tile
+            const bool have_part = SPLIT && kc != 0;
+            if (SPLIT && kc + chunk_blocks < k_pad) {
+                // not the last chunk of K: move the partial sums into registers (round-to-nearest adds) and
+                // hand the accumulator back
+#pragma unroll
+                for (int s4 = 0; s4 < (SPLIT ? 4 : 0); ++s4) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + col_part * (BN / COL_SPLIT) + s4 * 32, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        part[(s4 * 32 + i) % (SPLIT ? 128 : 1)] = (have_part ? part[(s4 * 32 + i) % (SPLIT ? 128 : 1)] : 0.0f) + __uint_as_float(r[i]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CG == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0));
+                    else         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
+                }
+                continue;
+            }
+#pragma unroll (SPLIT ? NBOX : 1)
+            for (int cc = 0; cc < NBOX; ++cc) {
+                const int c = col_part * NBOX + cc;
                 const int64_t col = col0 + (int64_t)c * CHUNK;
                 // A box that crosses the right edge is clipped by the TMA unit in 16-byte units: when the row
                 // length in bytes is not a multiple of 16 that last box is written with plain stores instead.
@@ -532,6 +568,11 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                         tc_wait_ld();
                     }
                     uint32_t (&r)[32] = rr[sub % PRE];
+                    if (have_part) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            r[i] = __float_as_uint(__uint_as_float(r[i]) + part[((cc * SUBS + sub) * 32 + i) % (SPLIT ? 128 : 1)]);
+                    }
                     float v[32];
                     if (p.sb_inv_vec) {                       // per-channel weight scales: one alpha per column
                         const int64_t scol_v = col + sub * 32;
@@ -610,6 +651,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 if (CG == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0));
                 else         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
             }
+          }
         }
         if (lane == 0) bulk_wait_all();                           // every store has reached global memory before exit
         if (warp == 2) { PROF_STORE(6, 7, -1) }
@@ -665,9 +707,9 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
 }
 
 // CTA-pair kernels launch as clusters of 2; the grid is one CTA per SM that can be paired.
-template <int CG, int OUT, int EPI_WARPS>
+template <int CG, int OUT, int EPI_WARPS, bool SPLIT = false>
 static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const Params& p, int64_t num_tiles, cudaStream_t st) {
-    auto k = k_gemm_fp8<CG, OUT, EPI_WARPS>;
+    auto k = k_gemm_fp8<CG, OUT, EPI_WARPS, SPLIT>;
     constexpr int THREADS = 64 + 32 * EPI_WARPS;
     // per device and cheap, so set on every launch rather than cached
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return FP8_ERR_CUDA;
@@ -697,8 +739,16 @@ static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
 }
 
 template <int CG>
-static fp8_status dispatch(int out_kind, bool short_k, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
+static fp8_status dispatch(int out_kind, bool short_k, bool split, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md,
                            const Params& p, int64_t num_tiles, cudaStream_t st) {
+    if (split && !short_k) {                                      // within one chunk of K there is nothing to split
+        switch (out_kind) {
+            case OUT_F32:  return launch<CG, OUT_F32, 8, true>(ma, mb, md, p, num_tiles, st);
+            case OUT_BF16: return launch<CG, OUT_BF16, 8, true>(ma, mb, md, p, num_tiles, st);
+            case OUT_E4M3: return launch<CG, OUT_E4M3, 8, true>(ma, mb, md, p, num_tiles, st);
+            default:       return launch<CG, OUT_E5M2, 8, true>(ma, mb, md, p, num_tiles, st);
+        }
+    }
     if (short_k) {
         switch (out_kind) {
             case OUT_F32:  return launch<CG, OUT_F32, 8>(ma, mb, md, p, num_tiles, st);
@@ -789,8 +839,9 @@ static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint
     p.idesc = (1u << 4) | ((uint32_t)d->fa << 7) | ((uint32_t)d->fb << 10) | ((a_mn ? 1u : 0u) << 15) |
               ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
     const bool short_k = (K + BK - 1) / BK <= SHORT_K_BLOCKS;
-    return cg == 2 ? dispatch<2>(out_kind, short_k, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st)
-                   : dispatch<1>(out_kind, short_k, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st);
+    const bool split = d->acc == FP8_ACC_SPLIT;
+    return cg == 2 ? dispatch<2>(out_kind, short_k, split, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st)
+                   : dispatch<1>(out_kind, short_k, split, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st);
 }
 
 }  // namespace gemm
@@ -802,7 +853,8 @@ extern "C" {
 
 static bool desc_enums_ok(const fp8_gemm_desc* d) {
     return (d->fa == FP8_E4M3 || d->fa == FP8_E5M2) && (d->fb == FP8_E4M3 || d->fb == FP8_E5M2) &&
-           (d->ma == FP8_MAJOR_K || d->ma == FP8_MAJOR_MN) && (d->mb == FP8_MAJOR_K || d->mb == FP8_MAJOR_MN);
+           (d->ma == FP8_MAJOR_K || d->ma == FP8_MAJOR_MN) && (d->mb == FP8_MAJOR_K || d->mb == FP8_MAJOR_MN) &&
+           (d->acc == FP8_ACC_FAST || d->acc == FP8_ACC_SPLIT);
 }
 
 fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,

@@ -51,6 +51,9 @@ def test_argument_errors_are_reported_before_any_launch():
     d.fa = 4
     assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 2
     d.fa = 0
+    d.acc = 2                                                                           # not an fp8_accumulate
+    assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 2
+    d.acc = api.ACC_SPLIT
     d.M = -1
     assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 3       # FP8_ERR_SHAPE
     d.M = 128
@@ -95,6 +98,11 @@ def test_argument_errors_of_the_wider_entry_points():
     assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 2, 0, one, one, one, None, None) == 2
     assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 0, 3, one, one, one, None, None) == 2
     assert lib.fp8_gemm_channel_scales(ctypes.byref(d), one, one, one, one, None, None, None) == 1
+    d.acc = 7
+    assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 0, 0, one, one, one, None, None) == 2
+    assert lib.fp8_gemm_channel_scales(ctypes.byref(d), one, one, one, one, one, None, None) == 2
+    assert lib.fp8_gemm_batched(ctypes.byref(d), 1, one, 0, one, 0, one, 0, one, one, None, None) == 2
+    d.acc = api.ACC_FAST
     assert lib.fp8_gemm_batched(ctypes.byref(d), -1, one, 0, one, 0, one, 0, one, one, None, None) == 3
     assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 100, one, 256 * 128, one, 256 * 256, one, one, None, None) == 3   # members overlap
     assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 256 * 128 + 8, one, 256 * 128, one, 256 * 256, one, one, None, None) == 4

@@ -36,7 +36,7 @@ def _pad_cols(a_np, mult=16, fill=0x7F):
     return buf
 
 
-def _run(A_np, fa, ma, B_np, fb, mb, M, N, K, out_dtype, sa_inv=0.013, sb_inv=0.5, want_amax=True):
+def _run(A_np, fa, ma, B_np, fb, mb, M, N, K, out_dtype, sa_inv=0.013, sb_inv=0.5, want_amax=True, acc=api.ACC_FAST):
     """A_np is the stored array ([M,K] or [K,M]); B_np the stored array ([N,K] or [K,N])."""
     A_buf, B_buf = _pad_cols(A_np), _pad_cols(B_np)
     A = torch.from_numpy(A_buf).to(DEV)[:, : A_np.shape[1]]
@@ -46,7 +46,7 @@ def _run(A_np, fa, ma, B_np, fb, mb, M, N, K, out_dtype, sa_inv=0.013, sb_inv=0.
     D_full = torch.full((M + 1, ldd), 777.0, dtype=out_dtype, device=DEV)       # guard row and pad columns
     D = D_full[:M, :N]
     amax = _scalar(-1.0) if want_amax else None
-    api.fp8_gemm(A, fa, ma, B, fb, mb, D, _scalar(sa_inv), _scalar(sb_inv), amax)
+    api.fp8_gemm(A, fa, ma, B, fb, mb, D, _scalar(sa_inv), _scalar(sb_inv), amax, acc=acc)
     torch.cuda.synchronize()
     st, detail = api.fp8_async_status()
     assert st == 0, "device-side wait expired, code %d" % detail
@@ -166,6 +166,111 @@ def test_same_sign_accumulation_bound():
         bound = 1e-5 if K <= 2048 else (K / 32) * 2.0 ** -23
         assert rel.max() <= bound, (K, rel.max(), bound)
         assert np.all(to_np_bits(D).astype(np.float64) <= ref * (1 + 2.0 ** -23))     # truncation never overshoots
+
+
+@pytest.mark.parametrize("M,K,ma,mb", [(128, 2048, api.MAJOR_K, api.MAJOR_K), (384, 2064, api.MAJOR_MN, api.MAJOR_MN),
+                                        (128, 4096, api.MAJOR_K, api.MAJOR_MN), (384, 6176, api.MAJOR_K, api.MAJOR_K),
+                                        (384, 16384, api.MAJOR_MN, api.MAJOR_MN), (128, 49152, api.MAJOR_K, api.MAJOR_K)])
+def test_split_accumulation_same_sign(M, K, ma, mb):
+    """ACC_SPLIT on all-positive operands (the accumulator's worst case): partial sums every 2048 of K are
+    added with round-to-nearest, so 1e-5 * sum|ab| holds at every K (M = 128: one CTA per tile; 384: CTA
+    pairs, the second pair half empty)"""
+    rng = np.random.default_rng(1000 + K + M)
+    N = 264
+    A_np = _codes(rng, E4, (M, K) if ma == api.MAJOR_K else (K, M), spread=1.0) & 0x7F
+    B_np = _codes(rng, E5, (N, K) if mb == api.MAJOR_K else (K, N), spread=1.0) & 0x7F
+    _run(A_np, E4, ma, B_np, E5, mb, M, N, K, torch.float32, sa_inv=1.0, sb_inv=1.0, acc=api.ACC_SPLIT)   # checks 1e-5 * sum|ab|
+    if K <= 6176:
+        _run(A_np, E4, ma, B_np, E5, mb, M, N, K, torch.bfloat16, sa_inv=1.0, sb_inv=1.0, acc=api.ACC_SPLIT)
+
+
+@pytest.mark.parametrize("M,N,K", [(129, 257, 2048 + 129), (300, 520, 4096 + 200), (128, 256, 8192), (1, 8, 2064)])
+@pytest.mark.parametrize("ma,mb", [(api.MAJOR_K, api.MAJOR_MN), (api.MAJOR_K, api.MAJOR_K), (api.MAJOR_MN, api.MAJOR_K)])
+def test_split_accumulation_mixed_sign_ragged(M, N, K, ma, mb):
+    """ACC_SPLIT on the usual mixed-sign codes: ragged M, N and K (a last chunk shorter than 2048, a last
+    K-block shorter than 128)"""
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+    A_np = _codes(rng, E5, (M, K) if ma == api.MAJOR_K else (K, M))
+    B_np = _codes(rng, E4, (N, K) if mb == api.MAJOR_K else (K, N))
+    _run(A_np, E5, ma, B_np, E4, mb, M, N, K, torch.float32, acc=api.ACC_SPLIT)
+    if mb == api.MAJOR_MN:
+        _run(A_np, E5, ma, B_np, E4, mb, M, N, K, torch.bfloat16, acc=api.ACC_SPLIT)
+
+
+def test_split_accumulation_many_tiles():
+    """more tile pairs than SM pairs with two chunks per tile: the two TMEM accumulators change owner
+    (chunk parity) from tile to tile"""
+    rng = np.random.default_rng(6)
+    M, N, K = 2600, 3904, 2304                   # 11 x 16 = 176 tile pairs
+    A_np = _codes(rng, E4, (M, K)) & 0x7F
+    B_np = _codes(rng, E4, (K, N)) & 0x7F
+    D = torch.empty(M, N, dtype=torch.float32, device=DEV)
+    amax = _scalar(0.0)
+    api.fp8_gemm(torch.from_numpy(A_np).to(DEV), E4, api.MAJOR_K, torch.from_numpy(B_np).to(DEV), E4, api.MAJOR_MN, D,
+                 _scalar(0.25), _scalar(0.125), amax, acc=api.ACC_SPLIT)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    t = oracle.decode_table(E4)
+    ref = (t[A_np] @ t[B_np]) * (0.25 * 0.125)   # all terms positive: ref is also sum|ab| (library fp64 matmul as reference)
+    got = to_np_bits(D)
+    assert (np.abs(got.astype(np.float64) - ref) / ref).max() < 1e-5
+    assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(got.reshape(-1))
+
+
+def test_split_equals_fast_up_to_2048():
+    """within one 2048-wide chunk both modes run the same additions: identical bits"""
+    rng = np.random.default_rng(5)
+    for K in (512, 1024, 1040, 2048):
+        M, N = 256, 512
+        A = torch.from_numpy(_codes(rng, E4, (M, K))).to(DEV)
+        B = torch.from_numpy(_codes(rng, E4, (N, K))).to(DEV)
+        D0 = torch.empty(M, N, dtype=torch.float32, device=DEV)
+        D1 = torch.empty_like(D0)
+        api.fp8_gemm(A, E4, api.MAJOR_K, B, E4, api.MAJOR_K, D0, _scalar(1.0), _scalar(1.0), acc=api.ACC_FAST)
+        api.fp8_gemm(A, E4, api.MAJOR_K, B, E4, api.MAJOR_K, D1, _scalar(1.0), _scalar(1.0), acc=api.ACC_SPLIT)
+        torch.cuda.synchronize()
+        assert torch.equal(D0.view(torch.int32), D1.view(torch.int32))
+
+
+def test_split_accumulation_other_entry_points():
+    """ACC_SPLIT through the FP8-output, per-channel-scale and batched entry points on all-positive codes at
+    K = 6144 + 64 (three full chunks and a short one)"""
+    rng = np.random.default_rng(4242)
+    M, N, K = 384, 520, 6144 + 64
+    A_np = _codes(rng, E4, (M, K), spread=1.0) & 0x7F
+    B_np = _codes(rng, E4, (N, K), spread=1.0) & 0x7F
+    A, B = torch.from_numpy(A_np).to(DEV), torch.from_numpy(B_np).to(DEV)
+    ref, sabs = oracle.gemm_rows(A_np, E4, (K, 1), B_np, E4, (1, K), N, K, 0, M, 0.5, 0.25, threads=THREADS)
+    # FP8 output
+    scale_d = float(oracle.scale_from_amax(np.float32(np.abs(ref).max()), E4)[0])
+    ldd = (N + 15) // 16 * 16
+    D8_full = torch.full((M + 1, ldd), 0xA5, dtype=torch.uint8, device=DEV)
+    amax = _scalar(-1.0)
+    api.fp8_gemm_fp8out(A, E4, api.MAJOR_K, B, E4, api.MAJOR_K, D8_full[:M, :N], E4, _scalar(0.5), _scalar(0.25), _scalar(scale_d),
+                        amax, acc=api.ACC_SPLIT)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    assert bool((D8_full[M:, :] == 0xA5).all()) and bool((D8_full[:M, N:] == 0xA5).all())
+    enc = lambda y: oracle.quantize(y.reshape(-1), 1.0, E4, threads=THREADS).reshape(y.shape)
+    assert check_gemm_fp8out(D8_full[:M, :N].cpu().numpy(), ref, sabs, scale_d, enc).all()
+    assert abs(amax.item() - np.abs(ref).max()) <= 1e-5 * np.abs(ref).max()
+    # per-channel inverse scales of B
+    sv = np.exp2(rng.integers(-3, 3, size=N)).astype(np.float32) * np.float32(0.3)
+    refc, sabsc = oracle.gemm_rows_colscale(A_np, E4, (K, 1), B_np, E4, (1, K), N, K, 0, M, 0.5, sv, threads=THREADS)
+    Dc = torch.empty(M, N, dtype=torch.float32, device=DEV)
+    api.fp8_gemm_channel_scales(A, E4, api.MAJOR_K, B, E4, api.MAJOR_K, Dc, _scalar(0.5), torch.from_numpy(sv).to(DEV), acc=api.ACC_SPLIT)
+    torch.cuda.synchronize()
+    assert (np.abs(to_np_bits(Dc).astype(np.float64) - refc) / sabsc).max() < 1e-5
+    # batched: three members, the same B for each, A rolled by member
+    Ab = torch.stack([A.roll(b, 0) for b in range(3)])
+    Bb = torch.stack([B, B, B])
+    Db = torch.empty(3, M, N, dtype=torch.float32, device=DEV)
+    api.fp8_gemm_batched(Ab, E4, api.MAJOR_K, Bb, E4, api.MAJOR_K, Db, _scalar(0.5), _scalar(0.25), acc=api.ACC_SPLIT)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    got = to_np_bits(Db).astype(np.float64)
+    for b in range(3):
+        assert (np.abs(got[b] - np.roll(ref, b, 0)) / np.roll(sabs, b, 0)).max() < 1e-5, b
 
 
 def test_many_tiles_persistent_schedule():
