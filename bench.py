@@ -296,6 +296,14 @@ def bench_next_rows(torch, api, synth, device, pk, iters=5):
     api.fp8_scales_from_amax(am, api.E4M3, sv, siv)
     ms = timed(lambda: api.fp8_quantize_channels(W, 0, api.E4M3, sv, Wq))
     out["quantize_channels_cols_W"] = {"ms": round(ms, 4), "gbs": round(3.0 * nW / ms / 1e6, 1), "frac_of_measured_hbm": round(3.0 * nW / ms / 1e6 / pk["hbm_gbs"], 4)}
+    # codes in both orientations from one pass (4 B per bf16 element): dY-shaped [8192 x 16384] and X-shaped [8192 x 4096]
+    for name, (r_, c_) in (("quantize_transpose_dY_8192x16384", (TOKENS, D_OUT)), ("quantize_transpose_X_8192x4096", (TOKENS, D_IN))):
+        xt = synth.gradients(r_ * c_, 4, device=device).view(r_, c_)
+        o1 = torch.empty(r_, c_, dtype=torch.uint8, device=device)
+        o2 = torch.empty(c_, r_, dtype=torch.uint8, device=device)
+        ms = timed(lambda: api.fp8_quantize_transpose(xt, api.E5M2, s, o1, o2, a))
+        out[name] = {"ms": round(ms, 4), "gbs": round(4.0 * r_ * c_ / ms / 1e6, 1), "frac_of_measured_hbm": round(4.0 * r_ * c_ / ms / 1e6 / pk["hbm_gbs"], 4)}
+        del xt, o1, o2
     # forward GEMM with per-channel weight scales, and with FP8 (E4M3) output
     X = synth.activations(TOKENS * D_IN, 3, device=device).view(TOKENS, D_IN)
     Xq = torch.empty(TOKENS, D_IN, dtype=torch.uint8, device=device)

@@ -237,6 +237,26 @@ fp8_status fp8_gemm_fp8out(const fp8_gemm_desc* d, const uint8_t* A, const uint8
                            float* amax_d_dev, void* stream);
 
 /*
+ * fp8_quantize_transpose — Sections 3 and 4.1: the same FP8 tensor is consumed by two matrix multiplies
+ * that contract over different axes (an activation by the forward product and by the weight-gradient
+ * product, an output gradient by both backward products), so its codes are produced once in both
+ * orientations:
+ *   code(r,c) = encode_f( binary32(x[r*ldx + c]) * scale )        conversion rules of fp8_quantize
+ *   out  [r*ldo + c] = code(r,c)        (rows x cols; `out` may be NULL: transposed copy only)
+ *   out_t[c*ldt + r] = code(r,c)        (cols x rows)
+ *   *amax_dev (nullable) OVERWRITTEN with amax of x, same pass (definition of fp8_amax).
+ * x is rows x cols, row-major, pitch ldx elements; ldo >= cols, ldt >= rows (bytes), else FP8_ERR_SHAPE.
+ * One pass: 128 x 128 tiles, transposed through shared memory, every global access a full 128-byte line.
+ * The tiled path needs rows and cols multiples of 4, x aligned to 4 elements with ldx a multiple of 4, and
+ * out / out_t / ldo / ldt multiples of 4 bytes; anything else takes an element-wise kernel with identical
+ * results.  rows*cols == 0 is a no-op (amax = 0).
+ */
+fp8_status fp8_quantize_transpose(const void* x, fp8_wide t, int64_t rows, int64_t cols, int64_t ldx,
+                                  fp8_format f, fp8_overflow o, const float* scale_dev,
+                                  uint8_t* out, int64_t ldo, uint8_t* out_t, int64_t ldt,
+                                  float* amax_dev, void* stream);
+
+/*
  * Per-channel scale factors — Section 4.2: post-training quantization uses "per-channel scaling factors for
  * weights, per-tensor scaling factors for activations".  A channel is a row or a column of a 2-D tensor
  * x (rows x cols, row-major, pitch ld elements): axis 0 = one channel per column, axis 1 = one per row.

@@ -23,7 +23,7 @@ ACC_FAST, ACC_SPLIT = 0, 1    # fp8_accumulate
 EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
            "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_fake_quantize",
            "fp8_scale_pow2_from_amax", "fp8_gemm", "fp8_gemm_fp8out", "fp8_amax_channels", "fp8_scales_from_amax",
-           "fp8_quantize_channels", "fp8_gemm_channel_scales", "fp8_gemm_batched",
+           "fp8_quantize_channels", "fp8_quantize_transpose", "fp8_gemm_channel_scales", "fp8_gemm_batched",
            "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
 
 
@@ -89,6 +89,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_scales_from_amax.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     lib.fp8_quantize_channels.restype = i32
     lib.fp8_quantize_channels.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, vp, vp, i64, vp]
+    lib.fp8_quantize_transpose.restype = i32
+    lib.fp8_quantize_transpose.argtypes = [vp, i32, i64, i64, i64, i32, i32, vp, vp, i64, vp, i64, vp, vp]
     lib.fp8_gemm_channel_scales.restype = i32
     lib.fp8_gemm_channel_scales.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.fp8_gemm_batched.restype = i32
@@ -290,6 +292,25 @@ def fp8_quantize_channels(x: torch.Tensor, axis: int, fmt: int, scale_vec: torch
     _check(load().fp8_quantize_channels(x.data_ptr(), _wide_of(x), rows, cols, ld, axis, fmt, overflow,
                                         _vec(scale_vec, cols if axis == 0 else rows, "scale_vec"), out.data_ptr(), ld_out, _stream()),
            "fp8_quantize_channels")
+
+
+def fp8_quantize_transpose(x: torch.Tensor, fmt: int, scale: torch.Tensor, out: torch.Tensor | None, out_t: torch.Tensor,
+                           amax_out: torch.Tensor | None = None, overflow: int = SATURATE) -> None:
+    """codes of the 2-D tensor x in both orientations from one pass: ``out`` [rows, cols] (or None) and
+    ``out_t`` [cols, rows]; ``amax_out`` optionally receives amax of x."""
+    rows, cols, ldx = _rows2d(x, "x")
+    trows, tcols, ldt = _rows2d(out_t, "out_t")
+    if out_t.dtype != torch.uint8 or (trows, tcols) != (cols, rows):
+        raise TypeError("out_t must be a uint8 tensor of the transposed shape of x")
+    ldo = 0
+    if out is not None:
+        orows, ocols, ldo = _rows2d(out, "out")
+        if out.dtype != torch.uint8 or (orows, ocols) != (rows, cols):
+            raise TypeError("out must be a uint8 tensor of the shape of x")
+    _check(load().fp8_quantize_transpose(x.data_ptr(), _wide_of(x), rows, cols, ldx, fmt, overflow, _scalar(scale, "scale"),
+                                         None if out is None else out.data_ptr(), ldo, out_t.data_ptr(), ldt,
+                                         None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()),
+           "fp8_quantize_transpose")
 
 
 def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,

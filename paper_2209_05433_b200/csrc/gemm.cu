@@ -264,18 +264,24 @@ constexpr int OUT_F32 = 0, OUT_BF16 = 1, OUT_E4M3 = 2, OUT_E5M2 = 3;
 // 32 accumulator values (already multiplied by alpha) -> 32 FP8 codes of y = v * scale_d, packed in 8 words.
 // Same rules as the cast kernels: hardware convert unless a special value (or, non-saturating, an overflow)
 // is present; a NaN code takes the sign of v.
+__device__ __forceinline__ float fmax_nan(float a, float b) {      // NaN if either operand is NaN
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
 template <int FMT>
 __device__ __forceinline__ void encode32(const float (&v)[32], float scale_d, bool nosat, uint32_t (&w)[8]) {
     float y[32];
-    float poison = 0.0f, top = 0.0f;
+    float top = 0.0f;                                             // max |y|, NaN if any y is NaN
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
         y[i] = v[i] * scale_d;
-        poison = fmaf(y[i], 0.0f, poison);
-        top = fmaxf(top, fabsf(y[i]));
+        top = fmax_nan(top, fabsf(y[i]));
     }
     const bool over = Fmt<FMT>::nosat_limit_inclusive ? top >= Fmt<FMT>::nosat_limit : top > Fmt<FMT>::nosat_limit;
-    if (poison == poison && !(nosat && over)) {
+    const bool finite = top <= 3.402823466e38f;                   // false for NaN and for Inf
+    if (finite && !(nosat && over)) {
 #pragma unroll
         for (int q = 0; q < 8; ++q) w[q] = cvt_quad<FMT>(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
     } else {
@@ -329,9 +335,16 @@ __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
            const __grid_constant__ CUtensorMap map_d, const Params p) {
     using G = Geo<CG>;
-    constexpr int EPI_BUFS = 8 / EPI_WARPS;
-    constexpr int STAGES = G::STAGES;
+    // Short K (eight epilogue warps, one accumulator per tile): the kernel is bound by its output stream, so
+    // two stages of the operand ring are given to the epilogue: three staging buffers per warp, whose TMA
+    // stores drain while the warp converts its next boxes.
+    constexpr bool SHORT = EPI_WARPS == 8 && !SPLIT;
+    constexpr int EPI_BUFS = SHORT ? 3 : 8 / EPI_WARPS;
+    constexpr int STAGES = SHORT ? G::STAGES - 2 : G::STAGES;
     constexpr uint32_t STAGE_BYTES = G::STAGE_BYTES;
+    constexpr uint32_t RING_BYTES = (uint32_t)STAGES * STAGE_BYTES;
+    static_assert(STAGES % G::FG == 0 && STAGES >= G::FG, "ring depth is a multiple of the stages consumed per wait");
+    static_assert(RING_BYTES + (uint32_t)(EPI_WARPS * EPI_BUFS) * EPI_BUF_BYTES <= SMEM_TILES + SMEM_EPI, "shared memory budget");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;                 // 1024-byte aligned tile ring
@@ -493,8 +506,9 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         const float sa_inv = __ldg(p.sa_inv);
         const float alpha = p.sb_inv_vec ? 0.0f : sa_inv * __ldg(p.sb_inv);
         const float scale_d = (OUT == OUT_E4M3 || OUT == OUT_E5M2) ? __ldg(p.scale_d) : 1.0f;
-        uint32_t running = 0;                                     // max of stored magnitude bits (bf16: 16-bit patterns)
-        const uint32_t epi_base = ring + SMEM_TILES + (uint32_t)(warp - 2) * (uint32_t)EPI_BUFS * EPI_BUF_BYTES;
+        uint32_t running = 0;                                     // bf16: max of stored 16-bit magnitude patterns, two lanes
+        float runf = 0.0f;                                        // fp32 / FP8 output: max |v|, NaN once any v is NaN
+        const uint32_t epi_base = ring + RING_BYTES + (uint32_t)(warp - 2) * (uint32_t)EPI_BUFS * EPI_BUF_BYTES;
         constexpr int COL_SPLIT = EPI_WARPS / 4;                  // warps sharing a lane quarter split the columns
         const int col_part = (warp - 2) >> 2;
         uint32_t buf = 0;
@@ -609,12 +623,12 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                                 for (int i = 0; i < 16; ++i) running = __vmaxu2(running, w[i] & 0x7FFF7FFFu);
                             } else {
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) running = max(running, __float_as_uint(v[i]) & 0x7FFFFFFFu);
+                                for (int i = 0; i < 32; ++i) runf = fmax_nan(runf, fabsf(v[i]));
                             }
                         } else {
                             for (int i = 0; i < 32 && scol + i < p.N; ++i) {
                                 if (OUT == OUT_BF16) running = __vmaxu2(running, ((i & 1) ? (w[i >> 1] >> 16) : w[i >> 1]) & 0x7FFFu);
-                                else                 running = max(running, __float_as_uint(v[i]) & 0x7FFFFFFFu);
+                                else                 runf = fmax_nan(runf, fabsf(v[i]));
                             }
                         }
                     }
@@ -656,7 +670,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         if (lane == 0) bulk_wait_all();                           // every store has reached global memory before exit
         if (warp == 2) { PROF_STORE(6, 7, -1) }
         if (p.amax_bits) {
-            uint32_t bits = OUT == OUT_BF16 ? (max(running & 0xFFFFu, running >> 16) << 16) : running;
+            uint32_t bits = OUT == OUT_BF16 ? (max(running & 0xFFFFu, running >> 16) << 16) : __float_as_uint(runf);
             bits = warp_max_u32(canonical_nan_bits(bits));
             if (lane == 0 && bits != 0u) atomicMax(p.amax_bits, bits);
         }

@@ -92,6 +92,15 @@ def test_argument_errors_of_the_wider_entry_points():
     assert lib.fp8_quantize_channels(one, 1, 4, 4, 4, 0, 0, 0, None, one, 4, None) == 1
     assert lib.fp8_quantize_channels(one, 1, 4, 4, 4, 0, 0, 0, one, one, 2, None) == 3
     assert lib.fp8_quantize_channels(one, 1, 4, 4, 4, 1, 4, 0, one, one, 4, None) == 2
+    # quantize + transposed copy
+    assert lib.fp8_quantize_transpose(one, 1, 4, 4, 4, 0, 0, one, one, 4, None, 4, None, None) == 1      # no out_t
+    assert lib.fp8_quantize_transpose(one, 1, 4, 4, 4, 0, 0, None, one, 4, one, 4, None, None) == 1      # no scale
+    assert lib.fp8_quantize_transpose(one, 3, 4, 4, 4, 0, 0, one, one, 4, one, 4, None, None) == 2
+    assert lib.fp8_quantize_transpose(one, 1, 4, 4, 4, 0, 2, one, one, 4, one, 4, None, None) == 2
+    assert lib.fp8_quantize_transpose(one, 1, 4, 8, 4, 0, 0, one, one, 8, one, 4, None, None) == 3       # ldx < cols
+    assert lib.fp8_quantize_transpose(one, 1, 4, 8, 8, 0, 0, one, one, 4, one, 4, None, None) == 3       # ldo < cols
+    assert lib.fp8_quantize_transpose(one, 1, 4, 8, 8, 0, 0, one, None, 0, one, 2, None, None) == 3      # ldt < rows
+    assert lib.fp8_quantize_transpose(None, 1, 0, 8, 8, 0, 0, one, None, 0, None, 0, None, None) == 0    # empty: nothing touched
     # GEMM variants
     d = api.GemmDesc(256, 256, 128, 0, 0, 0, 0, 128, 128, 256, 1)
     assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 0, 0, one, one, None, None, None) == 1
