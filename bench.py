@@ -233,6 +233,76 @@ def bench_cast_sweep(torch, api, synth, device, log2n, iters=20):
     return out
 
 
+def bench_cast_sizes(torch, api, synth, device, pk, sizes=(20, 24, 28, 30)):
+    """The bandwidth sweep over tensor sizes (bf16, 2^20 .. 2^30 elements).  Each kernel is timed twice:
+     - "same_buffer": 20 back-to-back calls on one tensor; below ~126 MB of traffic the tensor stays in L2, so the
+       figure is flagged l2_resident and is a latency / L2 number, not an HBM one;
+     - "ring": a CUDA graph of calls that walk a ring of distinct tensors totalling more than 512 MB, so that every
+       call misses L2: the HBM-honest figure for the small sizes (and the launch cost without host gaps)."""
+    out = {}
+    sc = torch.tensor([3.0, 1.0 / 3.0, 0.0, 0.0, 0.0], dtype=torch.float32, device=device)
+    s, si, a, s2, si2 = sc[0:1], sc[1:2], sc[2:3], sc[3:4], sc[4:5]
+    for log2n in sizes:
+        n = 1 << log2n
+        ring = max(1, -(-(640 << 20) // (2 * n)))            # tensors of 2n bytes totalling >= 640 MB
+        if log2n >= 30:
+            ring = 1                                         # 2 GB already
+        total = ring * n
+        x = synth.normal_laplace_mixture(total, 1, synth.T_ID, device=device)
+        codes = torch.empty(total, dtype=torch.uint8, device=device)
+        back = torch.empty(total, dtype=torch.bfloat16, device=device)
+        xs = [x[i * n:(i + 1) * n] for i in range(ring)]
+        cs = [codes[i * n:(i + 1) * n] for i in range(ring)]
+        bs = [back[i * n:(i + 1) * n] for i in range(ring)]
+        cases = {
+            "amax": (lambda i: api.fp8_amax(xs[i], a), 2.0 * n),
+            "quantize_e4m3_with_amax": (lambda i: api.fp8_quantize(xs[i], api.E4M3, s, cs[i], api.SATURATE, a), 3.0 * n),
+            "quantize_current_e4m3": (lambda i: api.fp8_quantize_current(xs[i], api.E4M3, cs[i], a, s2, si2), 5.0 * n),
+            "dequantize_e4m3": (lambda i: api.fp8_dequantize(cs[i], api.E4M3, si, bs[i]), 3.0 * n),
+        }
+        row = {"ring_tensors": ring}
+        for name, (fn, nbytes) in cases.items():
+            for _ in range(3):
+                fn(0)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(20):
+                fn(0)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / 20
+            entry = {"same_buffer": {"us": round(ms * 1e3, 2), "gbs": round(nbytes / ms / 1e6, 1), "l2_resident": bool(nbytes < (126 << 20))}}
+            calls = max(ring, 8)
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                for i in range(min(ring, 3)):
+                    fn(i)
+                side.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for i in range(calls):
+                        fn(i % ring)
+            torch.cuda.current_stream().wait_stream(side)
+            graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            gms = e0.elapsed_time(e1) / calls
+            entry["ring"] = {"us": round(gms * 1e3, 2), "gbs": round(nbytes / gms / 1e6, 1),
+                             "frac_of_measured_hbm": round(nbytes / gms / 1e6 / pk["hbm_gbs"], 4), "calls_in_graph": calls}
+            del graph
+            row[name] = entry
+        out["2pow%d" % log2n] = row
+        del x, codes, back, xs, cs, bs
+        torch.cuda.empty_cache()
+    return out
+
+
 def bench_gemm_alone(torch, step, seconds=2.0):
     """The forward GEMM of the step by itself: best single launch (burst) and a back-to-back loop of at
     least `seconds` (sustained, under the power cap)."""
@@ -456,6 +526,9 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.cast_sizes_only:
+        print(json.dumps({"cast_sizes": bench_cast_sizes(torch, api, synth, device, peaks())}))
+        return
     if args.next_rows_only:
         # profiling aid: only the kernels beyond the core path, each on workload-shaped tensors
         print(json.dumps({"next_rows": bench_next_rows(torch, api, synth, device, peaks(), iters=max(1, min(args.steps, 5)))}))
@@ -605,6 +678,7 @@ def run_ours(args):
             cast = bench_cast_sweep(torch, api, synth, device, args.cast_log2n)
             for v in cast.values():
                 v["frac_of_measured_hbm"] = round(v["gbs"] / pk["hbm_gbs"], 4)
+        cast_sizes = bench_cast_sizes(torch, api, synth, device, pk) if world == 1 and not args.no_cast_sweep else None
         gemm_alone = bench_gemm_alone(torch, step) if world == 1 and not args.no_next_rows else None
         next_rows = None
         if world == 1 and not args.no_next_rows:
@@ -627,6 +701,7 @@ def run_ours(args):
                     "how": "pinned host buffers; upload, kernels and download of consecutive steps overlap on three streams"},
             "gpu_launches": int(launches), "gpu_launches_note": "kernels plus 4-byte memset nodes enqueued by the library in the timed region",
             "roofline": roofline, "roofline_cast": roofline_cast, "kernels": kernels, "cast_sweep_2pow%d" % args.cast_log2n: cast,
+            "cast_sizes": cast_sizes,
             "gemm_alone": gemm_alone,
             "next_rows": next_rows,
             "cpu_baseline": cpu,
@@ -646,6 +721,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cast-sweep", action="store_true")
     ap.add_argument("--no-next-rows", action="store_true")
+    ap.add_argument("--cast-sizes-only", action="store_true", help="only the cast bandwidth sweep over 2^20 .. 2^30 elements")
     ap.add_argument("--next-rows-only", action="store_true", help="profiling aid: run only the next-row kernels")
     ap.add_argument("--cast-log2n", type=int, default=28)
     ap.add_argument("--unfused-cast", action="store_true", help="amax, scale and quantize as three calls per tensor instead of fp8_quantize_current")
