@@ -63,8 +63,9 @@ constexpr int UMMA_K = 32;          // K of one tcgen05.mma for 8-bit operands
 constexpr int MAX_STAGES = 6;
 constexpr int ACC_STAGES = 2;       // 2 x 256 columns = all 512 TMEM columns
 // Epilogue width: 4 warps with two staging buffers each (long K: the epilogue has slack, fewer resident warps
-// leave the MMA-issuing thread undisturbed) or 8 warps with one buffer each (short K: the kernel is bound by
-// its output stream; two warps per TMEM lane quarter split the tile's columns).
+// leave the MMA-issuing thread undisturbed) or 8 warps (short K: the kernel is bound by its output stream; two
+// warps per TMEM lane quarter split the tile's columns and each warp has three buffers, two ring stages' worth).
+// Split accumulation also runs 8 warps (one buffer each): its partial sums need 128 registers per thread.
 constexpr int SHORT_K_BLOCKS = 8;   // K <= 1024: eight epilogue warps
 constexpr int SPLIT_BLOCKS = 16;    // split accumulation: the TMEM accumulator is drained into registers every 2048 of K
 constexpr uint32_t A_BYTES = BM * BK;          // 16 KiB: this CTA's 128 rows of A
@@ -78,7 +79,7 @@ template <int CG> struct Geo {
 };
 constexpr uint32_t SMEM_TILES = 4 * (A_BYTES + BN * BK);            // = 6 * (A_BYTES + BN/2 * BK)
 constexpr uint32_t EPI_BUF_BYTES = 4096;                            // 32 rows x 128 B, one TMA store box
-constexpr uint32_t SMEM_EPI = 8 * EPI_BUF_BYTES;                    // staging buffers of the epilogue warps (4 x 2 or 8 x 1)
+constexpr uint32_t SMEM_EPI = 8 * EPI_BUF_BYTES;                    // staging buffers of the epilogue warps (4 x 2 or 8 x 1; short K adds two ring stages)
 constexpr uint32_t SMEM_BARRIERS = 256;
 constexpr uint32_t SMEM_BYTES = SMEM_TILES + SMEM_EPI + SMEM_BARRIERS + 1024;   // + slack to align the ring to 1024 B
 constexpr uint32_t TMEM_COLS = 512;
