@@ -99,6 +99,9 @@ def _linear_layer(seed, T, I, O, w_sigma, passes):
             dX = torch.empty(T, I, dtype=torch.bfloat16, device=DEV)
             api.fp8_gemm(Gq, api.E5M2, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, sig, siw, amax)
             _check_gemm(dX, amax, Gh, E5, (O, 1), Wh, E4, (1, O), O, wsig, wsiw, rng)
+            # the same product with split accumulation (partial sums every 2048 of K added in registers)
+            api.fp8_gemm(Gq, api.E5M2, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, sig, siw, amax, acc=api.ACC_SPLIT)
+            _check_gemm(dX, amax, Gh, E5, (O, 1), Wh, E4, (1, O), O, wsig, wsiw, rng)
             del dX
         if "wgrad" in passes:    # dW[I,O] = X^T . dY
             dW = torch.empty(I, O, dtype=torch.bfloat16, device=DEV)
