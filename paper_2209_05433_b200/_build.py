@@ -13,7 +13,7 @@ HEADERS = ["common.cuh", "codec.cuh", os.path.join("..", "..", "include", "fp8_b
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-    "-shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v",
+    "-shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v", "--threads", "2",
 ]
 
 

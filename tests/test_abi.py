@@ -116,3 +116,34 @@ def test_argument_errors_of_the_wider_entry_points():
     assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 100, one, 256 * 128, one, 256 * 256, one, one, None, None) == 3   # members overlap
     assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 256 * 128 + 8, one, 256 * 128, one, 256 * 256, one, one, None, None) == 4
     assert lib.fp8_gemm_batched(ctypes.byref(d), 70000, one, 256 * 128, one, 256 * 128, one, 256 * 256, one, one, None, None) == 5
+
+
+def test_header_is_plain_c_and_the_struct_layout_matches_the_binding(tmp_path):
+    """the boundary is a C ABI: the header compiles as C11 on its own, and a C program links against the
+    library by symbol name; sizes and offsets of fp8_gemm_desc equal those of the ctypes mirror"""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "abi_probe.c"
+    src.write_text(
+        '#include <stddef.h>\n#include <stdio.h>\n#include "fp8_b200.h"\n'
+        "int main(void) {\n"
+        "    fp8_gemm_desc d;\n"
+        '    printf("%zu %zu %zu %zu %zu %zu %zu\\n", sizeof d, offsetof(fp8_gemm_desc, K), offsetof(fp8_gemm_desc, fa),\n'
+        "           offsetof(fp8_gemm_desc, mb), offsetof(fp8_gemm_desc, lda), offsetof(fp8_gemm_desc, out), offsetof(fp8_gemm_desc, acc));\n"
+        '    printf("%s\\n", fp8_status_string(FP8_ERR_ALIGN));\n'
+        "    return fp8_amax(NULL, FP8_BF16, 4, NULL, NULL) == FP8_ERR_NULL ? 0 : 1;\n"
+        "}\n")
+    exe = tmp_path / "abi_probe"
+    lib_dir = os.path.dirname(api.library_path())
+    api.load()                                  # builds the library if it is missing
+    subprocess.check_call([gcc, "-std=c11", "-Wall", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"), str(src),
+                           "-o", str(exe), "-L", lib_dir, "-l:libfp8_b200.so", "-Wl,-rpath," + lib_dir])
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, out.stderr
+    sizes, msg = out.stdout.strip().split("\n")
+    G = api.GemmDesc
+    assert [int(v) for v in sizes.split()] == [ctypes.sizeof(G), G.K.offset, G.fa.offset, G.mb.offset, G.lda.offset, G.out.offset, G.acc.offset]
+    assert msg == "operand not 16-byte aligned"
