@@ -127,7 +127,8 @@ def _brute_force_encode(y32, fmt, overflow):
     # (E4M3: 480 at mantissa 111; E5M2: 2^16 in the next binade)
     virtual = 480.0 if fmt == E4M3 else 65536.0
     ext = np.concatenate([mags, [virtual]])
-    y = y32.astype(np.float64)
+    with np.errstate(invalid="ignore"):       # signalling NaN patterns among the inputs
+        y = y32.astype(np.float64)
     a = np.abs(y)
     sign = (y32.view(np.uint32) >> 31).astype(np.uint8) << 7
     out = np.zeros(y.shape, dtype=np.uint8)
