@@ -334,15 +334,20 @@ def bench_next_rows(torch, api, synth, device, pk, iters=5):
     """The rows beyond the core path, each timed alone on workload-shaped tensors: simulated-FP8 round trip,
     per-channel weight scales, FP8-output GEMM, attention-style batched GEMM."""
     def timed(fn):
+        """mean of `iters` groups of 4 back-to-back calls (launch gaps overlap the previous call, as inside a step);
+        a short idle first, so that each kernel is timed alone and not in the power state its predecessor left"""
+        torch.cuda.synchronize()
+        time.sleep(0.25)
         for _ in range(3):
             fn()
-        times = []
-        for _ in range(iters):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(); fn(); e1.record()
-            torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1))
-        return statistics.median(times)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(4 * iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (4 * iters)
 
     out = {}
     f32 = torch.float32
