@@ -292,8 +292,10 @@ fp8_status fp8_gemm_channel_scales(const fp8_gemm_desc* d, const uint8_t* A, con
  * attention batched matrix multiplies)".  `batch` independent products with the same shape, layouts,
  * formats and per-tensor scales (one scale for the whole batched tensor), in one launch:
  *   D_b = (A_b . B_b) * (sa_inv * sb_inv),   A_b = A + b*stride_a, B_b = B + b*stride_b, D_b = D + b*stride_d
- * Strides are in elements of the respective tensor, at least one whole matrix apart, and 16-byte aligned
- * (in bytes).  amax_d_dev (optional) receives the amax over all batch members.  batch == 0 is a no-op
+ * Strides are in elements of the respective tensor and 16-byte aligned (in bytes).  The members of D lie at
+ * least one whole matrix apart (they are written); the members of A and of B are only read, so any positive
+ * stride is accepted: members may interleave (heads stored side by side inside a row, slices of K of one
+ * matrix) or overlap.  amax_d_dev (optional) receives the amax over all batch members.  batch == 0 is a no-op
  * (amax = 0); batch <= 65535.  Everything else as fp8_gemm.
  */
 fp8_status fp8_gemm_batched(const fp8_gemm_desc* d, int64_t batch,

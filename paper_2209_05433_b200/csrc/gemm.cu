@@ -806,8 +806,8 @@ static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint
         }
         if ((reinterpret_cast<uintptr_t>(D) & 15u) || ((d->ldd * esz) & 15)) return FP8_ERR_ALIGN;
         if (bt.count > 1) {
-            const int64_t a_rows = a_mn ? K : M, b_rows_total = b_mn ? K : N;
-            if (bt.stride_a < a_rows * d->lda || bt.stride_b < b_rows_total * d->ldb || bt.stride_d < M * d->ldd) return FP8_ERR_SHAPE;
+            // written members may not overlap; read-only members may interleave or overlap
+            if (bt.stride_a <= 0 || bt.stride_b <= 0 || bt.stride_d < M * d->ldd) return FP8_ERR_SHAPE;
             if ((bt.stride_a & 15) || (bt.stride_b & 15) || ((bt.stride_d * esz) & 15)) return FP8_ERR_ALIGN;
         }
         if (tiles_m * tiles_n * (bt.count > 0 ? bt.count : 1) > (int64_t)1 << 30 || M > ((int64_t)1 << 31) - 256 ||

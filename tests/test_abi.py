@@ -113,7 +113,8 @@ def test_argument_errors_of_the_wider_entry_points():
     assert lib.fp8_gemm_batched(ctypes.byref(d), 1, one, 0, one, 0, one, 0, one, one, None, None) == 2
     d.acc = api.ACC_FAST
     assert lib.fp8_gemm_batched(ctypes.byref(d), -1, one, 0, one, 0, one, 0, one, one, None, None) == 3
-    assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 100, one, 256 * 128, one, 256 * 256, one, one, None, None) == 3   # members overlap
+    assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 256 * 128, one, 256 * 128, one, 100, one, one, None, None) == 3   # members of D overlap
+    assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 0, one, 256 * 128, one, 256 * 256, one, one, None, None) == 3
     assert lib.fp8_gemm_batched(ctypes.byref(d), 4, one, 256 * 128 + 8, one, 256 * 128, one, 256 * 256, one, one, None, None) == 4
     assert lib.fp8_gemm_batched(ctypes.byref(d), 70000, one, 256 * 128, one, 256 * 128, one, 256 * 256, one, one, None, None) == 5
 

@@ -437,3 +437,28 @@ def test_batched_gemm(case, out_dtype):
     a2 = _scalar(-1.0)
     api.fp8_amax(D.contiguous(), a2)
     assert amax.cpu().numpy().view(np.uint32)[0] == a2.cpu().numpy().view(np.uint32)[0]
+
+
+def test_batched_gemm_interleaved_heads():
+    """attention heads stored side by side inside a row ([S, H, d] tensors): the batch stride of the read-only
+    operands is the head width, smaller than a matrix; scores = Q_h . K_h^T for every head in one launch"""
+    rng = np.random.default_rng(17)
+    S, H, Dh = 200, 5, 64
+    Q_np = _codes(rng, E4, (S, H * Dh))
+    K_np = _codes(rng, E4, (S, H * Dh))
+    Q = torch.from_numpy(Q_np).to(DEV).view(S, H, Dh).permute(1, 0, 2)        # [H, S, Dh] view, strides (Dh, H*Dh, 1)
+    Kt = torch.from_numpy(K_np).to(DEV).view(S, H, Dh).permute(1, 0, 2)
+    ldd = 200
+    D = torch.empty(H, S, ldd, dtype=torch.float32, device=DEV)[:, :, :S]
+    amax = _scalar(-1.0)
+    api.fp8_gemm_batched(Q, E4, api.MAJOR_K, Kt, E4, api.MAJOR_K, D, _scalar(0.25), _scalar(0.5), amax)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    got = to_np_bits(D)
+    for h in range(H):
+        qa = np.ascontiguousarray(Q_np[:, h * Dh:(h + 1) * Dh])
+        ka = np.ascontiguousarray(K_np[:, h * Dh:(h + 1) * Dh])
+        ref, sabs = oracle.gemm_rows(qa, E4, (Dh, 1), ka, E4, (1, Dh), S, Dh, 0, S, 0.25, 0.5, threads=THREADS)
+        ok, worst = check_gemm_f32(got[h], ref, sabs)
+        assert ok.all(), (h, worst)
+    assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(got.reshape(-1))

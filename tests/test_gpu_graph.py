@@ -64,3 +64,54 @@ def test_step_replays_from_a_cuda_graph(fused):
         assert api.fp8_async_status()[0] == 0
         for k in graph_buf:
             assert torch.equal(graph_buf[k].view(torch.uint8), eager_buf[k].view(torch.uint8)), (k, trial)
+
+
+def test_rows_beyond_the_core_path_replay_from_a_cuda_graph():
+    """quantize + transposed copy, the K-major weight-gradient GEMM on the transposed codes with split
+    accumulation, an FP8-output GEMM and a batched GEMM, captured once and replayed on new values"""
+    T, I, O = 2304, 256, 384                      # the weight gradient contracts over T = 2304: two chunks of K
+    X = synth.activations(T * I, 5, device=DEV).view(T, I)
+    dY = synth.gradients(T * O, 6, device=DEV).view(T, O)
+    u8, f32 = torch.uint8, torch.float32
+
+    def buffers():
+        return {"Xq": torch.empty(T, I, dtype=u8, device=DEV), "XqT": torch.empty(I, T, dtype=u8, device=DEV),
+                "Gq": torch.empty(T, O, dtype=u8, device=DEV), "GqT": torch.empty(O, T, dtype=u8, device=DEV),
+                "dW": torch.empty(I, O, dtype=f32, device=DEV), "dWq": torch.empty(I, O, dtype=u8, device=DEV),
+                "P": torch.empty(3, I, O, dtype=torch.bfloat16, device=DEV), "scal": torch.zeros(8, dtype=f32, device=DEV)}
+
+    sx, sg = torch.tensor([2.0], device=DEV), torch.tensor([4096.0], device=DEV)
+    six, sig, sd = torch.tensor([0.5], device=DEV), torch.tensor([1.0 / 4096.0], device=DEV), torch.tensor([8.0], device=DEV)
+
+    def step(b):
+        s = b["scal"]
+        api.fp8_quantize_transpose(X, api.E4M3, sx, b["Xq"], b["XqT"], s[0:1])
+        api.fp8_quantize_transpose(dY, api.E5M2, sg, b["Gq"], b["GqT"], s[1:2])
+        api.fp8_gemm(b["XqT"], api.E4M3, api.MAJOR_K, b["GqT"], api.E5M2, api.MAJOR_K, b["dW"], six, sig, s[2:3], acc=api.ACC_SPLIT)
+        api.fp8_gemm_fp8out(b["XqT"], api.E4M3, api.MAJOR_K, b["GqT"], api.E5M2, api.MAJOR_K, b["dWq"], api.E4M3, six, sig, sd, s[3:4],
+                            acc=api.ACC_SPLIT)
+        A3 = b["XqT"].view(I, 3, T // 3).permute(1, 0, 2)          # three K-slices as batch members (pitched views)
+        B3 = b["GqT"].view(O, 3, T // 3).permute(1, 0, 2)
+        api.fp8_gemm_batched(A3, api.E4M3, api.MAJOR_K, B3, api.E5M2, api.MAJOR_K, b["P"], six, sig, s[4:5])
+
+    gb, eb = buffers(), buffers()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step(gb)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            step(gb)
+    torch.cuda.synchronize()
+    for trial in range(2):
+        X.copy_(synth.activations(T * I, 50 + trial, device=DEV).view(T, I))
+        dY.copy_(synth.gradients(T * O, 60 + trial, device=DEV).view(T, O) * (2.0 + trial))
+        g.replay()
+        step(eb)
+        torch.cuda.synchronize()
+        assert api.fp8_async_status()[0] == 0
+        for k in gb:
+            assert torch.equal(gb[k].view(u8), eb[k].view(u8)), (k, trial)
+    # the three K-slices add up to the whole weight-gradient product (bf16 partial results, loose check)
+    total = eb["P"].float().sum(0)
+    assert torch.allclose(total, eb["dW"], rtol=2e-2, atol=2e-2 * float(eb["dW"].abs().max()))
