@@ -198,8 +198,9 @@ fp8_status fp8_scale_pow2_from_amax(const float* amax_dev, fp8_format f,
  * Accumulation (`acc`): the products are exact and the tensor core adds them, 32 of K at a time, into a
  * binary32 accumulator whose additions round toward zero.
  *   FP8_ACC_FAST   one accumulator over all of K.  The error is below 1e-5 * sum_k|a.b| for K <= 2048 on any
- *                  data, and for any K when the products are mixed in sign (training tensors); products of
- *                  one sign lose up to (K/32) * 2^-23 of their sum.
+ *                  data; on products of mixed sign (training tensors) it grows slowly with K (measured 1.4e-7
+ *                  at K = 49152 on the workloads' tensors, 1.2e-5 at K = 2^20 on heavy-tailed codes); products
+ *                  of one sign lose up to (K/32) * 2^-23 of their sum.
  *   FP8_ACC_SPLIT  the accumulator is drained every 2048 of K and the partial sums are added in registers
  *                  with round-to-nearest: below 1e-5 * sum_k|a.b| for any data and any K, at a cost of a few
  *                  per cent of throughput.  Identical to FAST for K <= 2048.
