@@ -613,7 +613,10 @@ __global__ void k_scale_pow2_from_amax(const float* amax_dev, float fmax, float*
 // (8 bf16 / 4 f32) and every fourth row of the block's slab; per-column maxima stay separate inside the
 // packed words.  The four row lanes meet in shared memory, then one atomicMax per column per block.
 // amax_bits[cols] must be zero before.
-constexpr int kColsTx = 64, kColsTy = 4;
+#ifndef FP8_COLS_MIN_ROWS
+#define FP8_COLS_MIN_ROWS 256
+#endif
+constexpr int kColsTx = 64, kColsTy = 4, kColsUnroll = 8;       // 64 x 4 threads, eight row loads in flight per thread
 template <int WIDE>
 __global__ void __launch_bounds__(kColsTx * kColsTy)
 k_amax_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, int64_t rows_per_slab, uint32_t* amax_bits) {
@@ -638,12 +641,12 @@ k_amax_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, 
     };
     if (live) {
         int64_t r = r0 + ty;
-        for (; r + 3 * kColsTy < r1; r += 4 * kColsTy) {
-            uint4 v[4];
+        for (; r + (kColsUnroll - 1) * kColsTy < r1; r += kColsUnroll * kColsTy) {
+            uint4 v[kColsUnroll];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = ld_nc_v4(base + (r + u * kColsTy) * ld * ESZ);
+            for (int u = 0; u < kColsUnroll; ++u) v[u] = ld_nc_v4(base + (r + u * kColsTy) * ld * ESZ);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) fold(v[u]);
+            for (int u = 0; u < kColsUnroll; ++u) fold(v[u]);
         }
         for (; r < r1; r += kColsTy) fold(ld_nc_v4(base + r * ld * ESZ));
     }
@@ -1135,14 +1138,14 @@ static int grid_for(int64_t work_items) {
     return (int)g;
 }
 
-// rows per slab of the column kernels: about 16 blocks per SM in all, at least 64 rows (16 per thread)
+// rows per slab of the column kernels: about 16 blocks per SM in all, but at least 256 rows (64 per thread)
 static int64_t slab_rows(int64_t rows, int64_t col_blocks) {
     const int64_t want_blocks = (int64_t)sm_count() * 16;
     int64_t slabs = (want_blocks + col_blocks - 1) / col_blocks;
     if (slabs < 1) slabs = 1;
     int64_t per = (rows + slabs - 1) / slabs;
     per = (per + 15) / 16 * 16;
-    if (per < 64) per = 64;
+    if (per < FP8_COLS_MIN_ROWS) per = FP8_COLS_MIN_ROWS;          // short slabs are all launch, tail and atomics
     while ((rows + per - 1) / per > 65535) per *= 2;
     return per;
 }
