@@ -670,24 +670,43 @@ k_amax_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, 
     }
 }
 
-// AXIS 1, vector path: one warp per row.
+// AXIS 1, vector path.  A row is cut into segments of 32 lanes x kRowsUnroll 16-byte items; a warp takes one
+// (row, segment) unit at a time with all its loads in flight, so short-and-wide and tall-and-narrow tensors both
+// fill the GPU.  One unit per row: the warp stores the row's amax; several: atomicMax onto a zeroed vector.
+constexpr int kRowsUnroll = 4;
+constexpr int kRowsAmaxUnroll = 8;
+// amax: a unit is a row's span of `span` items (a multiple of 32 x kRowsAmaxUnroll), `segs` spans per row
 template <int WIDE>
 __global__ void __launch_bounds__(kThreads)
-k_amax_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, uint32_t* amax_bits) {
+k_amax_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, int64_t segs, int64_t span, uint32_t* amax_bits) {
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
     constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
     const int64_t n_warps = ((int64_t)gridDim.x * kThreads) >> 5;
     const int64_t n_items = cols / EPI;
-    for (int64_t r = warp; r < rows; r += n_warps) {
+    for (int64_t u = warp; u < rows * segs; u += n_warps) {
+        const int64_t r = u / segs, seg = u - r * segs;
         const char* row = reinterpret_cast<const char*>(x) + r * ld * ESZ;
+        const int64_t end = min(n_items, (seg + 1) * span);
+        int64_t i = seg * span + lane;
         uint32_t m = 0;
-        for (int64_t i = lane; i < n_items; i += 32) m = fold_abs_max<WIDE>(m, ld_nc_v4(row + i * 16));
+        for (; i + 32 * (kRowsAmaxUnroll - 1) < end; i += 32 * kRowsAmaxUnroll) {
+            uint4 v[kRowsAmaxUnroll];
+#pragma unroll
+            for (int k = 0; k < kRowsAmaxUnroll; ++k) v[k] = ld_nc_v4(row + (i + 32 * k) * 16);
+#pragma unroll
+            for (int k = 0; k < kRowsAmaxUnroll; ++k) m = fold_abs_max<WIDE>(m, v[k]);
+        }
+        for (; i < end; i += 32) m = fold_abs_max<WIDE>(m, ld_nc_v4(row + i * 16));
         m = finish_abs_max<WIDE>(m);
-        for (int64_t c = n_items * EPI + lane; c < cols; c += 32) m = max(m, canonical_nan_bits(scalar_abs_bits<WIDE>(row, c)));
+        if (seg == segs - 1)                                          // ragged tail of the row
+            for (int64_t c = n_items * EPI + lane; c < cols; c += 32) m = max(m, canonical_nan_bits(scalar_abs_bits<WIDE>(row, c)));
         m = warp_max_u32(m);
-        if (lane == 0) amax_bits[r] = m;
+        if (lane == 0) {
+            if (segs == 1) amax_bits[r] = m;
+            else if (m) atomicMax(&amax_bits[r], m);
+        }
     }
 }
 
@@ -776,10 +795,10 @@ k_quantize_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t 
     for (; r < r1; r += kColsTy) emit(r, ld_nc_v4(base + r * ld * ESZ));
 }
 
-// AXIS 1, vector path: one warp per row, the row's scale in a register.
+// AXIS 1, vector path: a warp per (row, segment) unit as in k_amax_rows, the row's scale in a register.
 template <int WIDE, int FMT, bool NOSAT>
 __global__ void __launch_bounds__(kThreads)
-k_quantize_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, const float* __restrict__ scale,
+k_quantize_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, int64_t segs, const float* __restrict__ scale,
                 uint8_t* __restrict__ out, int64_t ld_out) {
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
     constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
@@ -787,18 +806,30 @@ k_quantize_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t 
     const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
     const int64_t n_warps = ((int64_t)gridDim.x * kThreads) >> 5;
     const int64_t n_items = cols / EPI;
-    for (int64_t r = warp; r < rows; r += n_warps) {
+    auto emit = [&](uint8_t* orow, int64_t i, const uint4& v, float s) {
+        if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(orow) + i, quantize_item_bf16<FMT, NOSAT>(v, s));
+        else                   st_out(reinterpret_cast<uint32_t*>(orow) + i, quantize_item_f32<FMT, NOSAT>(v, s));
+    };
+    for (int64_t u = warp; u < rows * segs; u += n_warps) {
+        const int64_t r = u / segs, seg = u - r * segs;
         const float s = __ldg(scale + r);
         const char* row = reinterpret_cast<const char*>(x) + r * ld * ESZ;
         uint8_t* orow = out + r * ld_out;
-        for (int64_t i = lane; i < n_items; i += 32) {
-            const uint4 v = ld_nc_v4(row + i * 16);
-            if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(orow) + i, quantize_item_bf16<FMT, NOSAT>(v, s));
-            else                   st_out(reinterpret_cast<uint32_t*>(orow) + i, quantize_item_f32<FMT, NOSAT>(v, s));
+        const int64_t i0 = seg * (32 * kRowsUnroll) + lane;
+        if (i0 + 32 * (kRowsUnroll - 1) < n_items) {
+            uint4 v[kRowsUnroll];
+#pragma unroll
+            for (int k = 0; k < kRowsUnroll; ++k) v[k] = ld_nc_v4(row + (i0 + 32 * k) * 16);
+#pragma unroll
+            for (int k = 0; k < kRowsUnroll; ++k) emit(orow, i0 + 32 * k, v[k], s);
+        } else {
+            for (int64_t i = i0; i < n_items; i += 32) emit(orow, i, ld_nc_v4(row + i * 16), s);
         }
-        for (int64_t c = n_items * EPI + lane; c < cols; c += 32) {
-            const float xf = scalar_load<WIDE>(row, c);
-            orow[c] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * s, __float_as_uint(xf));
+        if (seg == segs - 1) {
+            for (int64_t c = n_items * EPI + lane; c < cols; c += 32) {
+                const float xf = scalar_load<WIDE>(row, c);
+                orow[c] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * s, __float_as_uint(xf));
+            }
         }
     }
 }
@@ -1138,6 +1169,13 @@ static int grid_for(int64_t work_items) {
     return (int)g;
 }
 
+// segments per row of the row kernels: 32 lanes x kRowsUnroll items each, at least one
+static int64_t row_segments(int64_t n_items) {
+    const int64_t per = 32 * kRowsUnroll;
+    const int64_t segs = (n_items + per - 1) / per;
+    return segs < 1 ? 1 : segs;
+}
+
 // rows per slab of the column kernels: about 16 blocks per SM in all, but at least 256 rows (64 per thread)
 static int64_t slab_rows(int64_t rows, int64_t col_blocks) {
     const int64_t want_blocks = (int64_t)sm_count() * 16;
@@ -1156,8 +1194,22 @@ static fp8_status launch_amax_channels(const void* x, int64_t rows, int64_t cols
     constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
     const int64_t channels = axis == 0 ? cols : rows;
     const bool vec = aligned16(x) && ((ld * ESZ) & 15) == 0;
-    if (axis == 1 && vec) {                                         // every row written exactly once: no zeroing needed
-        k_amax_rows<WIDE><<<grid_for(rows * 32), kThreads, 0, st>>>(x, rows, cols, ld, bits);
+    if (axis == 1 && vec) {
+        // spans per row: enough units for about four warps' worth per resident warp, no span shorter than one unrolled pass
+        const int64_t n_items = cols / EPI, pass = 32 * kRowsAmaxUnroll;
+        const int64_t want_units = (int64_t)sm_count() * 8 * (kThreads / 32) * 4;
+        int64_t segs = (want_units + rows - 1) / rows;
+        const int64_t max_segs = (n_items + pass - 1) / pass;
+        if (segs > max_segs) segs = max_segs;
+        if (segs < 1) segs = 1;
+        const int64_t span = ((n_items + segs - 1) / segs + pass - 1) / pass * pass;
+        segs = span > 0 ? (n_items + span - 1) / span : 1;
+        if (segs < 1) segs = 1;
+        if (segs > 1) {                                             // several warps share a row: atomicMax onto zeros
+            if (cudaMemsetAsync(bits, 0, (size_t)channels * 4, st) != cudaSuccess) return FP8_ERR_CUDA;
+            count_launches(1);
+        }
+        k_amax_rows<WIDE><<<grid_for(rows * segs * 32), kThreads, 0, st>>>(x, rows, cols, ld, segs, span, bits);
         count_launches(1);
         return launch_status();
     }
@@ -1184,7 +1236,8 @@ static fp8_status launch_quantize_channels(const void* x, int64_t rows, int64_t 
     constexpr int ESZ = WIDE == kWideBF16 ? 2 : 4;
     const bool vec = aligned16(x) && ((ld * ESZ) & 15) == 0 && (reinterpret_cast<uintptr_t>(out) & (EPI - 1)) == 0 && (ld_out % EPI) == 0;
     if (vec && axis == 1) {
-        k_quantize_rows<WIDE, FMT, NOSAT><<<grid_for(rows * 32), kThreads, 0, st>>>(x, rows, cols, ld, scale, out, ld_out);
+        const int64_t segs = row_segments(cols / EPI);
+        k_quantize_rows<WIDE, FMT, NOSAT><<<grid_for(rows * segs * 32), kThreads, 0, st>>>(x, rows, cols, ld, segs, scale, out, ld_out);
         count_launches(1);
         return launch_status();
     }

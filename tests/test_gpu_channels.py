@@ -21,7 +21,7 @@ def _scalar(v):
 @pytest.mark.parametrize("wide", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("axis", [0, 1])
 @pytest.mark.parametrize("shape,pitch", [((1, 1), 1), ((37, 53), 53), ((64, 128), 128), ((300, 520), 528), ((1024, 4096), 4096),
-                                          ((5, 4099), 4099), ((513, 72), 80)])
+                                          ((5, 4099), 4099), ((513, 72), 80), ((3, 16405), 16416), ((2000, 264), 264), ((700, 1300), 1312)])
 def test_amax_scales_quantize_per_channel(wide, axis, shape, pitch):
     rows, cols = shape
     base = synth.weights(rows * pitch + 8, 13, 0.02, dtype=wide, device=DEV)
