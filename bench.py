@@ -402,6 +402,18 @@ def bench_next_rows(torch, api, synth, device, pk, iters=5):
     out["gemm_dgrad_same_codes_one_accumulator"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
     del dX
     del W, X, Y, Yq
+    # a weight-bandwidth-bound product with few output tiles: 16 rows against W^T stored [4096 x 16384] (K = 16384),
+    # plain and with the contraction cut into slices
+    Xs = torch.randint(0, 0x78, (16, D_OUT), dtype=torch.uint8, device=device)
+    Wt = torch.randint(0, 0x78, (D_IN, D_OUT), dtype=torch.uint8, device=device)          # [N = 4096, K = 16384], K-major
+    Ys = torch.empty(16, D_IN, dtype=torch.bfloat16, device=device)
+    sp, nb = api.fp8_gemm_splitk_workspace(16, D_IN, D_OUT)
+    ws = torch.empty(max(nb // 4, 4), dtype=f32, device=device)
+    ms = timed(lambda: api.fp8_gemm(Xs, api.E4M3, api.MAJOR_K, Wt, api.E4M3, api.MAJOR_K, Ys, si, si, a))
+    out["gemm_16x4096x16384_one_launch"] = {"ms": round(ms, 4), "weight_gbs": round(D_IN * D_OUT / ms / 1e6, 1)}
+    ms = timed(lambda: api.fp8_gemm_splitk(Xs, api.E4M3, api.MAJOR_K, Wt, api.E4M3, api.MAJOR_K, Ys, si, si, ws if nb else None, a))
+    out["gemm_16x4096x16384_splitk"] = {"ms": round(ms, 4), "weight_gbs": round(D_IN * D_OUT / ms / 1e6, 1), "splits": sp}
+    del Xs, Wt, Ys, ws
     # attention-style batched products: 32 heads, 4096 tokens, head dim 128: scores = Q.K^T, context = P.V
     H, S, Dh = 32, 4096, 128
     Q = torch.randint(0, 0x78, (H, S, Dh), dtype=torch.uint8, device=device)

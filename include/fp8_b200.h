@@ -306,6 +306,27 @@ fp8_status fp8_gemm_batched(const fp8_gemm_desc* d, int64_t batch,
                             float* amax_d_dev, void* stream);
 
 /*
+ * fp8_gemm_splitk — fp8_gemm for problems with few output tiles and a long contraction (a weight-bandwidth-
+ * bound product of a few rows with a wide weight matrix): K is cut into `splits` slices that run as members of
+ * one batched launch, each writing an fp32 partial product (already multiplied by sa_inv * sb_inv) into the
+ * caller's workspace, and a second kernel adds the partials in slice order, rounds to `out` and records amax.
+ *   D[i,j] = round_out( sum_s fl32( (sum_{k in slice s} a.b) * (sa_inv * sb_inv) ) )
+ * Same tolerance as fp8_gemm (the extra binary32 roundings are ~1e-7 relative).  Deterministic.
+ * fp8_gemm_splitk_workspace reports, for a descriptor, the number of slices the library will use on the
+ * current device and the workspace it needs: splits = 1 (bytes = 0) whenever a cost model of the kernel (operand
+ * bytes over min(tiles x 90 GB/s, HBM), plus the second launch and the partials) predicts less than 15 % gain,
+ * K < 2048, N is not a multiple of 4, or K does not divide into slices that are multiples of 256; then
+ * fp8_gemm_splitk is exactly fp8_gemm.  Otherwise splits is a power of two up to 16 and
+ * bytes = splits * M * N * 4.  workspace_dev: 16-byte aligned device memory of at least that size (else
+ * FP8_ERR_ALIGN / FP8_ERR_SHAPE), owned by the caller, contents undefined afterwards.  With splits > 1, D needs
+ * only element alignment and ldd >= N.
+ */
+fp8_status fp8_gemm_splitk_workspace(const fp8_gemm_desc* d, int* splits_out, size_t* bytes_out);
+fp8_status fp8_gemm_splitk(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,
+                           const float* scale_inv_a_dev, const float* scale_inv_b_dev, float* amax_d_dev,
+                           void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/*
  * fp8_async_status — reads and clears the device-side error latch of the
  * current device (synchronises the device).  FP8_OK, or FP8_ERR_TIMEOUT if a
  * kernel gave up on a bounded wait since the last call; *detail (optional, host

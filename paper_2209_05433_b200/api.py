@@ -24,6 +24,7 @@ EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_curr
            "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_fake_quantize",
            "fp8_scale_pow2_from_amax", "fp8_gemm", "fp8_gemm_fp8out", "fp8_amax_channels", "fp8_scales_from_amax",
            "fp8_quantize_channels", "fp8_quantize_transpose", "fp8_gemm_channel_scales", "fp8_gemm_batched",
+           "fp8_gemm_splitk", "fp8_gemm_splitk_workspace",
            "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
 
 
@@ -95,6 +96,10 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_gemm_channel_scales.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp]
     lib.fp8_gemm_batched.restype = i32
     lib.fp8_gemm_batched.argtypes = [ctypes.POINTER(GemmDesc), i64, vp, i64, vp, i64, vp, i64, vp, vp, vp, vp]
+    lib.fp8_gemm_splitk_workspace.restype = i32
+    lib.fp8_gemm_splitk_workspace.argtypes = [ctypes.POINTER(GemmDesc), ctypes.POINTER(ctypes.c_int), ctypes.POINTER(sz)]
+    lib.fp8_gemm_splitk.restype = i32
+    lib.fp8_gemm_splitk.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.fp8_async_status.restype = i32
     lib.fp8_async_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
     lib.fp8_status_string.restype = ctypes.c_char_p
@@ -237,6 +242,40 @@ def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: in
     _check(load().fp8_gemm(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
                            _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
                            None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()), "fp8_gemm")
+
+
+def _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc):
+    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
+        raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D tensor")
+    for t, name in ((A, "A"), (B, "B"), (D, "D")):
+        if not t.is_cuda or t.stride(1) != 1:
+            raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
+    M, K = (A.shape[0], A.shape[1]) if ma == MAJOR_K else (A.shape[1], A.shape[0])
+    Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
+    if K != Kb or tuple(D.shape) != (M, N):
+        raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
+    return GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D), acc)
+
+
+def fp8_gemm_splitk_workspace(M: int, N: int, K: int) -> tuple[int, int]:
+    """(number of K-slices, workspace bytes) fp8_gemm_splitk uses for this shape on the current device"""
+    d = GemmDesc(M, N, K, E4M3, E4M3, MAJOR_K, MAJOR_K, K, K, N, BF16, ACC_FAST)
+    splits, nbytes = ctypes.c_int(0), ctypes.c_size_t(0)
+    _check(load().fp8_gemm_splitk_workspace(ctypes.byref(d), ctypes.byref(splits), ctypes.byref(nbytes)), "fp8_gemm_splitk_workspace")
+    return splits.value, nbytes.value
+
+
+def fp8_gemm_splitk(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
+                    scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, workspace: torch.Tensor | None,
+                    amax_out: torch.Tensor | None = None, acc: int = ACC_FAST) -> None:
+    """fp8_gemm with the contraction cut into slices when the problem has few output tiles; ``workspace`` is a
+    CUDA tensor of at least fp8_gemm_splitk_workspace(M, N, K)[1] bytes (None when that is 0)."""
+    d = _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc)
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (workspace.data_ptr(), workspace.numel() * workspace.element_size())
+    _check(load().fp8_gemm_splitk(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
+                                  _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
+                                  None if amax_out is None else _scalar(amax_out, "amax_out"), ws_ptr, ws_bytes, _stream()),
+           "fp8_gemm_splitk")
 
 
 def fp8_gemm_fp8out(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor, fd: int,

@@ -859,6 +859,82 @@ static fp8_status gemm_impl(const fp8_gemm_desc* d, const uint8_t* A, const uint
                    : dispatch<1>(out_kind, short_k, split, map_a, map_b, map_d, p, tiles_m * tiles_n * bt.count, st);
 }
 
+// ---- split-K for problems with few output tiles --------------------------------------------
+
+// Sum of `splits` fp32 partial products (already multiplied by alpha), rounded to the output type, with the
+// amax of the stored values.  Four columns per thread; the additions run in slice order, so the result does
+// not depend on the launch shape.
+template <int OUT>
+__global__ void __launch_bounds__(256)
+k_splitk_reduce(const float* __restrict__ part, int splits, int64_t M, int64_t N, void* __restrict__ D, int64_t ldd,
+                uint32_t* amax_bits) {
+    __shared__ uint32_t red[32];
+    const int64_t quads_per_row = (N + 3) / 4;
+    const int64_t total = M * quads_per_row;
+    const int64_t plane = M * N;
+    uint32_t running = 0;
+    for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < total; q += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = q / quads_per_row, j = (q - i * quads_per_row) * 4;
+        const int n = (int)min((int64_t)4, N - j);
+        float v[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        const float* p = part + i * N + j;
+        if (n == 4 && (N & 3) == 0) {
+            for (int sidx = 0; sidx < splits; ++sidx) {
+                const float4 t = *reinterpret_cast<const float4*>(p + (int64_t)sidx * plane);
+                v[0] += t.x; v[1] += t.y; v[2] += t.z; v[3] += t.w;
+            }
+        } else {
+            for (int sidx = 0; sidx < splits; ++sidx)
+                for (int e = 0; e < n; ++e) v[e] += p[(int64_t)sidx * plane + e];
+        }
+        if (OUT == OUT_F32) {
+            float* d = reinterpret_cast<float*>(D) + i * ldd + j;
+            for (int e = 0; e < n; ++e) {
+                d[e] = v[e];
+                running = max(running, canonical_nan_bits(__float_as_uint(v[e]) & 0x7FFFFFFFu));
+            }
+        } else {
+            uint16_t* d = reinterpret_cast<uint16_t*>(D) + i * ldd + j;
+            const uint32_t w0 = pack_bf16(v[0], v[1]), w1 = pack_bf16(v[2], v[3]);
+            const uint16_t h[4] = {(uint16_t)w0, (uint16_t)(w0 >> 16), (uint16_t)w1, (uint16_t)(w1 >> 16)};
+            for (int e = 0; e < n; ++e) {
+                d[e] = h[e];
+                running = max(running, canonical_nan_bits(((uint32_t)h[e] & 0x7FFFu) << 16));
+            }
+        }
+    }
+    if (amax_bits) block_atomic_max_bits(running, red, amax_bits);
+}
+
+// Number of K-slices for a problem.  Measured on B200: one output tile (a CTA, or a CTA pair) streams its operand
+// panels at about 90 GB/s (its ring of stages in flight over the memory latency), so a product with T tiles reads
+// its operands at min(T x 90 GB/s, HBM); slices multiply T, and cost a second launch plus the fp32 partials
+// (about 9 us + 8 B per partial element).  The smallest power of two (at most 16, slices multiples of 256 of K
+// and at least 1024 long, tiles x slices within the SMs) whose modelled time is at least 15 % below the
+// unsliced one is taken; 1 otherwise.
+static int choose_splits(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K < 2048 || (N & 3) != 0) return 1;    // fp32 partial rows are whole 16-byte units
+    const int cg = M > BM ? 2 : 1;
+    const double tiles = (double)(((M + BM * cg - 1) / (BM * cg)) * ((N + BN - 1) / BN));
+    const double workers = (double)(sm_count() / cg);
+    const double bytes = (double)K * (double)(M + N);
+    const double tile_rate = 90e9, hbm_rate = 6.0e12, split_cost = 9e-6, partial_rate = 5.0e12;
+    auto modelled = [&](int sl) {
+        double rate = tiles * sl * tile_rate;
+        if (rate > hbm_rate) rate = hbm_rate;
+        return bytes / rate + (sl > 1 ? split_cost + 8.0 * sl * (double)M * (double)N / partial_rate : 0.0);
+    };
+    const double base = modelled(1);
+    int best = 1;
+    double best_t = base;
+    for (int sl = 2; sl <= 16; sl *= 2) {
+        if (tiles * sl > workers || K % ((int64_t)sl * 256) != 0 || K / sl < 1024) break;
+        const double t = modelled(sl);
+        if (t < 0.95 * best_t) { best = sl; best_t = t; }
+    }
+    return best_t <= 0.85 * base ? best : 1;
+}
+
 }  // namespace gemm
 }  // namespace fp8b200
 
@@ -908,6 +984,62 @@ fp8_status fp8_gemm_fp8out(const fp8_gemm_desc* d, const uint8_t* A, const uint8
     if (!desc_enums_ok(d) || (fd != FP8_E4M3 && fd != FP8_E5M2) || (od != FP8_SATURATE && od != FP8_NOSAT)) return FP8_ERR_ENUM;
     return gemm_impl(d, A, B, D, fd == FP8_E4M3 ? OUT_E4M3 : OUT_E5M2, od == FP8_NOSAT ? 1 : 0, scale_inv_a_dev, scale_inv_b_dev,
                      nullptr, scale_d_dev, amax_d_dev, (cudaStream_t)stream);
+}
+
+fp8_status fp8_gemm_splitk_workspace(const fp8_gemm_desc* d, int* splits_out, size_t* bytes_out) {
+    using namespace fp8b200::gemm;
+    if (!d || !splits_out || !bytes_out) return FP8_ERR_NULL;
+    if (d->M < 0 || d->N < 0 || d->K < 0) return FP8_ERR_SHAPE;
+    const int s = choose_splits(d->M, d->N, d->K);
+    *splits_out = s;
+    *bytes_out = s > 1 ? (size_t)s * (size_t)d->M * (size_t)d->N * sizeof(float) : 0;
+    return FP8_OK;
+}
+
+fp8_status fp8_gemm_splitk(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, void* D,
+                           const float* scale_inv_a_dev, const float* scale_inv_b_dev, float* amax_d_dev,
+                           void* workspace_dev, size_t workspace_bytes, void* stream) {
+    using namespace fp8b200::gemm;
+    if (!d || !scale_inv_a_dev || !scale_inv_b_dev) return FP8_ERR_NULL;
+    if (!desc_enums_ok(d) || (d->out != FP8_F32 && d->out != FP8_BF16)) return FP8_ERR_ENUM;
+    const int out_kind = d->out == FP8_BF16 ? OUT_BF16 : OUT_F32;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int splits = (d->M >= 0 && d->N >= 0 && d->K >= 0) ? choose_splits(d->M, d->N, d->K) : 1;
+    if (splits == 1)
+        return gemm_impl(d, A, B, D, out_kind, 0, scale_inv_a_dev, scale_inv_b_dev, nullptr, nullptr, amax_d_dev, st);
+    const size_t need = (size_t)splits * (size_t)d->M * (size_t)d->N * sizeof(float);
+    if (!workspace_dev || !D) return FP8_ERR_NULL;
+    if (workspace_bytes < need) return FP8_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 15u) return FP8_ERR_ALIGN;
+    const int64_t esz = out_kind == OUT_F32 ? 4 : 2;
+    if (d->ldd < d->N) return FP8_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(D) & (uintptr_t)(esz - 1)) != 0) return FP8_ERR_ALIGN;
+    // the K-slices as members of one batched product with fp32 output (alpha applied per slice)
+    const int64_t ks = d->K / splits;
+    fp8_gemm_desc slice = *d;
+    slice.K = ks;
+    slice.ldd = d->N;
+    slice.out = FP8_F32;
+    const bool a_mn = d->ma == FP8_MAJOR_MN, b_mn = d->mb == FP8_MAJOR_MN;
+    Batch bt{splits, a_mn ? ks * d->lda : ks, b_mn ? ks * d->ldb : ks, d->M * d->N};
+    fp8_status rc = gemm_impl(&slice, A, B, workspace_dev, OUT_F32, 0, scale_inv_a_dev, scale_inv_b_dev, nullptr, nullptr, nullptr, st, bt);
+    if (rc != FP8_OK) return rc;
+    if (amax_d_dev) {
+        if (cudaMemsetAsync(amax_d_dev, 0, 4, st) != cudaSuccess) return FP8_ERR_CUDA;
+        count_launches(1);
+    }
+    const int64_t quads = d->M * ((d->N + 3) / 4);
+    int64_t grid = (quads + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 8;
+    if (grid > cap) grid = cap;
+    if (out_kind == OUT_F32)
+        k_splitk_reduce<OUT_F32><<<(unsigned)grid, 256, 0, st>>>(reinterpret_cast<const float*>(workspace_dev), splits, d->M, d->N, D, d->ldd,
+                                                                  reinterpret_cast<uint32_t*>(amax_d_dev));
+    else
+        k_splitk_reduce<OUT_BF16><<<(unsigned)grid, 256, 0, st>>>(reinterpret_cast<const float*>(workspace_dev), splits, d->M, d->N, D, d->ldd,
+                                                                   reinterpret_cast<uint32_t*>(amax_d_dev));
+    count_launches(1);
+    return launch_status();
 }
 
 #ifdef FP8_GEMM_PROFILE

@@ -107,7 +107,11 @@ def test_argument_errors_of_the_wider_entry_points():
     assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 2, 0, one, one, one, None, None) == 2
     assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 0, 3, one, one, one, None, None) == 2
     assert lib.fp8_gemm_channel_scales(ctypes.byref(d), one, one, one, one, None, None, None) == 1
+    # split-K: null outputs, enum and shape checks come before any device work
+    assert lib.fp8_gemm_splitk_workspace(ctypes.byref(d), None, None) == 1
+    assert lib.fp8_gemm_splitk(None, one, one, one, one, one, None, None, 0, None) == 1
     d.acc = 7
+    assert lib.fp8_gemm_splitk(ctypes.byref(d), one, one, one, one, one, None, None, 0, None) == 2
     assert lib.fp8_gemm_fp8out(ctypes.byref(d), one, one, one, 0, 0, one, one, one, None, None) == 2
     assert lib.fp8_gemm_channel_scales(ctypes.byref(d), one, one, one, one, one, None, None) == 2
     assert lib.fp8_gemm_batched(ctypes.byref(d), 1, one, 0, one, 0, one, 0, one, one, None, None) == 2

@@ -462,3 +462,69 @@ def test_batched_gemm_interleaved_heads():
         ok, worst = check_gemm_f32(got[h], ref, sabs)
         assert ok.all(), (h, worst)
     assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(got.reshape(-1))
+
+
+# ------------------------------------------------------------------ split-K (few output tiles) --
+
+@pytest.mark.parametrize("M,N,K", [(16, 2048, 16384), (128, 1024, 8192), (200, 512, 4096), (1, 256, 65536), (64, 260, 4096)])
+@pytest.mark.parametrize("ma,mb", [(api.MAJOR_K, api.MAJOR_K), (api.MAJOR_K, api.MAJOR_MN), (api.MAJOR_MN, api.MAJOR_K)])
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_splitk_gemm(M, N, K, ma, mb, out_dtype):
+    """a few rows against a wide weight matrix: K is cut into slices (the library says how many), partial
+    products are summed in slice order; same tolerance as fp8_gemm, amax of the stored output, guard bands"""
+    rng = np.random.default_rng(M + N + K)
+    A_np = _codes(rng, E5, (M, K) if ma == api.MAJOR_K else (K, M), spread=3.0)
+    B_np = _codes(rng, E4, (N, K) if mb == api.MAJOR_K else (K, N), spread=3.0)
+    A_buf, B_buf = _pad_cols(A_np), _pad_cols(B_np)                # row pitches that are multiples of 16 bytes
+    A = torch.from_numpy(A_buf).to(DEV)[:, : A_np.shape[1]]
+    B = torch.from_numpy(B_buf).to(DEV)[:, : B_np.shape[1]]
+    splits, nbytes = api.fp8_gemm_splitk_workspace(M, N, K)
+    assert splits >= 1 and nbytes == (splits * M * N * 4 if splits > 1 else 0)
+    if (M, N, K) != (64, 260, 4096):
+        assert splits > 1, "these shapes leave most SMs idle without slices"
+    ws = torch.full((nbytes // 4 + 64,), float("nan"), dtype=torch.float32, device=DEV)
+    ldd = N + 3                                                   # only element alignment is needed with slices
+    if splits == 1:
+        esz = 2 if out_dtype == torch.bfloat16 else 4
+        ldd = (N * esz + 15) // 16 * 16 // esz
+    D_full = torch.full((M + 1, ldd), 777.0, dtype=out_dtype, device=DEV)
+    D = D_full[:M, :N]
+    amax = _scalar(-1.0)
+    api.fp8_gemm_splitk(A, E5, ma, B, E4, mb, D, _scalar(0.013), _scalar(0.5), ws[: nbytes // 4] if nbytes else None, amax)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    assert bool((D_full[M:, :] == 777.0).all()) and bool((D_full[:M, N:] == 777.0).all()), "wrote outside D"
+    assert bool(torch.isnan(ws[nbytes // 4:]).all()), "wrote past the workspace"
+    a_str = (A_buf.shape[1], 1) if ma == api.MAJOR_K else (1, A_buf.shape[1])
+    b_str = (1, B_buf.shape[1]) if mb == api.MAJOR_K else (B_buf.shape[1], 1)
+    ref, sabs = oracle.gemm_rows(A_buf, E5, a_str, B_buf, E4, b_str, N, K, 0, M, 0.013, 0.5, threads=THREADS)
+    got = to_np_bits(D)
+    if out_dtype == torch.float32:
+        ok, worst = check_gemm_f32(got, ref, sabs)
+    else:
+        ok, _ = check_gemm_bf16(got, ref, sabs, oracle.round_bf16_from_f64)
+    assert ok.all(), np.argwhere(~ok)[:4].tolist()
+    a2 = _scalar(-1.0)
+    api.fp8_amax(D.contiguous(), a2)
+    assert amax.cpu().numpy().view(np.uint32)[0] == a2.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(got.reshape(-1))
+
+
+def test_splitk_workspace_errors_and_large_problems_take_the_plain_path():
+    assert api.fp8_gemm_splitk_workspace(8192, 16384, 4096) == (1, 0)       # tiles fill the GPU: no slices
+    assert api.fp8_gemm_splitk_workspace(16, 4096, 1024) == (1, 0)          # short contraction
+    assert api.fp8_gemm_splitk_workspace(16, 4098, 16384) == (1, 0)         # N not a multiple of 4
+    M, N, K = 16, 2048, 8192
+    splits, nbytes = api.fp8_gemm_splitk_workspace(M, N, K)
+    assert splits > 1
+    A = torch.zeros(M, K, dtype=torch.uint8, device=DEV)
+    B = torch.zeros(N, K, dtype=torch.uint8, device=DEV)
+    D = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+    one = _scalar(1.0)
+    with pytest.raises(api.Fp8Error, match="status 1"):
+        api.fp8_gemm_splitk(A, E4, api.MAJOR_K, B, E4, api.MAJOR_K, D, one, one, None)
+    small = torch.empty(nbytes // 4 - 4, dtype=torch.float32, device=DEV)
+    with pytest.raises(api.Fp8Error, match="status 3"):
+        api.fp8_gemm_splitk(A, E4, api.MAJOR_K, B, E4, api.MAJOR_K, D, one, one, small)
+    odd = torch.empty(nbytes // 4 + 4, dtype=torch.float32, device=DEV)[1:]
+    with pytest.raises(api.Fp8Error, match="status 4"):
+        api.fp8_gemm_splitk(A, E4, api.MAJOR_K, B, E4, api.MAJOR_K, D, one, one, odd)
