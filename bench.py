@@ -303,6 +303,90 @@ def bench_cast_sizes(torch, api, synth, device, pk, sizes=(20, 24, 28, 30)):
     return out
 
 
+def bench_config(torch, api, synth, device, pk, which):
+    """One of the five named workloads, every call timed alone (20 back-to-back launches after a short idle):
+    1 = 256 x 256 fp32 tensors, casts and a 256^3 GEMM (latency-bound); 2 = the cast size sweep; 3 = hidden-4096
+    forward (casts of X and W, forward GEMM); 4 = hidden-4096 backward (cast of dY, dgrad, wgrad); 5 = the
+    175B-class FFN, hidden 12288 (casts of X, W, dY; forward and dgrad GEMMs)."""
+    if which == 2:
+        return bench_cast_sizes(torch, api, synth, device, pk)
+
+    def timed(fn, n=20):
+        torch.cuda.synchronize()
+        time.sleep(0.25)
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    bf, f32, u8 = torch.bfloat16, torch.float32, torch.uint8
+    E4, E5, KM, MN = api.E4M3, api.E5M2, api.MAJOR_K, api.MAJOR_MN
+    out = {}
+
+    def cast(name, x, fmt):
+        q = torch.empty(x.shape, dtype=u8, device=device)
+        s = torch.zeros(3, dtype=f32, device=device)
+        esz = x.element_size()
+        ms = timed(lambda: api.fp8_quantize_current(x, fmt, q, s[0:1], s[1:2], s[2:3]))
+        nbytes = (2 * esz + 1.0) * x.numel()
+        out["quantize_current_" + name] = {"ms": round(ms, 4), "gbs": round(nbytes / ms / 1e6, 1),
+                                           "frac_of_measured_hbm": round(nbytes / ms / 1e6 / pk["hbm_gbs"], 4)}
+        return q, s[2:3]
+
+    def gemm(name, A, fa, ma, B, fb, mb, M, N, K, si_a, si_b, dtype=bf, n=20):
+        D = torch.empty(M, N, dtype=dtype, device=device)
+        am = torch.zeros(1, dtype=f32, device=device)
+        ms = timed(lambda: api.fp8_gemm(A, fa, ma, B, fb, mb, D, si_a, si_b, am), n)
+        tf = 2.0 * M * N * K / ms / 1e9
+        out["gemm_" + name] = {"ms": round(ms, 4), "tflops": round(tf, 1), "frac_of_2x_measured_bf16_burst": round(tf / (2 * pk["bf16_burst"]), 4),
+                               "frac_of_nominal_4500": round(tf / 4500.0, 4)}
+
+    if which == 1:
+        A = synth.normal_with_scaled_outliers(256 * 256, 0, synth.A_ID, 0.005, 64.0, dtype=f32, device=device).view(256, 256)
+        B = synth.normal_with_scaled_outliers(256 * 256, 0, synth.B_ID, 0.005, 64.0, dtype=f32, device=device).view(256, 256)
+        Aq, sia = cast("A_256x256_fp32", A, E4)
+        Bq, sib = cast("B_256x256_fp32", B, E4)
+        gemm("256x256x256_fp32_out", Aq, E4, KM, Bq, E4, KM, 256, 256, 256, sia, sib, dtype=f32)
+    elif which in (3, 4):
+        T, I, O = TOKENS, D_IN, D_OUT
+        X = synth.activations(T * I, 3, device=device).view(T, I)
+        W = synth.weights(I * O, 3, W_SIGMA, device=device).view(I, O)
+        Xq, six = cast("X_8192x4096", X, E4)
+        Wq, siw = cast("W_4096x16384", W, E4)
+        del X, W
+        if which == 3:
+            gemm("fprop_8192x16384x4096", Xq, E4, KM, Wq, E4, MN, T, O, I, six, siw)
+        else:
+            dY = synth.gradients(T * O, 4, device=device).view(T, O)
+            Gq, sig = cast("dY_8192x16384", dY, E5)
+            del dY
+            gemm("dgrad_8192x4096x16384", Gq, E5, KM, Wq, E4, KM, T, I, O, sig, siw)
+            gemm("wgrad_4096x16384x8192", Xq, E4, MN, Gq, E5, MN, I, O, T, six, sig)
+    elif which == 5:
+        T, I, O = 8192, 12288, 49152
+        X = synth.activations(T * I, 5, device=device).view(T, I)
+        Xq, six = cast("X_8192x12288", X, E4)
+        del X
+        W = synth.weights(I * O, 5, 0.006, device=device).view(I, O)
+        Wq, siw = cast("W_12288x49152", W, E4)
+        del W
+        dY = synth.gradients(T * O, 5, device=device).view(T, O)
+        Gq, sig = cast("dY_8192x49152", dY, E5)
+        del dY
+        torch.cuda.empty_cache()
+        gemm("fprop_8192x49152x12288", Xq, E4, KM, Wq, E4, MN, T, O, I, six, siw, n=5)
+        gemm("dgrad_8192x12288x49152", Gq, E5, KM, Wq, E4, KM, T, I, O, sig, siw, n=5)
+    else:
+        raise SystemExit("--config takes 1..5")
+    return out
+
+
 def bench_gemm_alone(torch, step, seconds=2.0):
     """The forward GEMM of the step by itself: best single launch (burst) and a back-to-back loop of at
     least `seconds` (sustained, under the power cap)."""
@@ -546,6 +630,9 @@ def run_ours(args):
     if args.cast_sizes_only:
         print(json.dumps({"cast_sizes": bench_cast_sizes(torch, api, synth, device, peaks())}))
         return
+    if args.config:
+        print(json.dumps({"config": args.config, "results": bench_config(torch, api, synth, device, peaks(), args.config)}))
+        return
     if args.next_rows_only:
         # profiling aid: only the kernels beyond the core path, each on workload-shaped tensors
         print(json.dumps({"next_rows": bench_next_rows(torch, api, synth, device, peaks(), iters=max(1, min(args.steps, 5)))}))
@@ -739,6 +826,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cast-sweep", action="store_true")
     ap.add_argument("--no-next-rows", action="store_true")
+    ap.add_argument("--config", type=int, default=0, help="run one of the five named workloads (1..5), every call timed alone")
     ap.add_argument("--cast-sizes-only", action="store_true", help="only the cast bandwidth sweep over 2^20 .. 2^30 elements")
     ap.add_argument("--next-rows-only", action="store_true", help="profiling aid: run only the next-row kernels")
     ap.add_argument("--cast-log2n", type=int, default=28)
