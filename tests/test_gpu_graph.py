@@ -115,3 +115,30 @@ def test_rows_beyond_the_core_path_replay_from_a_cuda_graph():
     # the three K-slices add up to the whole weight-gradient product (bf16 partial results, loose check)
     total = eb["P"].float().sum(0)
     assert torch.allclose(total, eb["dW"], rtol=2e-2, atol=2e-2 * float(eb["dW"].abs().max()))
+
+
+def test_two_streams_run_independent_steps_concurrently():
+    """two steps on two streams at once (separate buffers, separate current-scaling workspaces): each gives
+    what it gives alone"""
+    T, I, O = 640, 512, 768
+    inputs = []
+    for k in range(2):
+        inputs.append((synth.activations(T * I, 70 + k, device=DEV).view(T, I), synth.weights(I * O, 70 + k, 0.02, device=DEV).view(I, O),
+                       synth.gradients(T * O, 80 + k, device=DEV).view(T, O)))
+    alone = []
+    for X, W, dY in inputs:
+        b = _buffers(T, I, O)
+        _step(X, W, dY, b, True)
+        alone.append(b)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    together = [_buffers(T, I, O), _buffers(T, I, O)]
+    for rep in range(5):
+        for k, st in enumerate(streams):
+            with torch.cuda.stream(st):
+                _step(*inputs[k], together[k], True)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    for k in range(2):
+        for name in alone[k]:
+            assert torch.equal(alone[k][name].view(torch.uint8), together[k][name].view(torch.uint8)), (k, name)
