@@ -1,0 +1,165 @@
+"""Randomised shapes, layouts, formats, pitches, output types and accumulation modes through the GEMM entry
+points.  The reference is the plain definition evaluated with library routines: the oracle's decode table
+indexed by the codes, then a binary64 matrix product on the device (exact for E4M3 x E4M3, within 1e-12 of
+sum|a.b| otherwise), with sum|a.b| from the product of the absolute values.  Fixed seeds: the cases are the same
+on every run."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2209_05433_b200 import api
+from tests._util import check_gemm_bf16, check_gemm_f32, to_np_bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+TABLES = {}
+
+
+def _table(fmt):
+    if fmt not in TABLES:
+        TABLES[fmt] = torch.from_numpy(oracle.decode_table(fmt)).to(DEV)
+    return TABLES[fmt]
+
+
+def _operand(rng, rows, cols, fmt):
+    """finite random codes in a buffer whose pitch is a multiple of 16 plus a random number of 16-byte pads;
+    the padding holds NaN codes, so that a read outside the logical extent poisons the result"""
+    pitch = (cols + 15) // 16 * 16 + 16 * int(rng.integers(0, 3))
+    top = 0x7E if fmt == oracle.E4M3 else 0x7B
+    buf = np.full((rows, pitch), 0x7F, dtype=np.uint8)
+    buf[:, :cols] = rng.integers(0, top + 1, size=(rows, cols), dtype=np.uint8) | (rng.integers(0, 2, size=(rows, cols), dtype=np.uint8) << 7)
+    t = torch.from_numpy(buf).to(DEV)
+    return t[:, :cols]
+
+
+def _reference(A, fa, ma, B, fb, mb, alpha):
+    a = _table(fa)[A.long()]
+    b = _table(fb)[B.long()]
+    a = a if ma == api.MAJOR_K else a.t()                 # [M, K]
+    b = b.t() if mb == api.MAJOR_K else b                 # [K, N]
+    ref = (a @ b) * alpha
+    sabs = (a.abs() @ b.abs()) * alpha
+    return ref.cpu().numpy(), sabs.cpu().numpy()
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_gemm_case(seed):
+    rng = np.random.default_rng(9000 + seed)
+    big = seed % 6 == 0
+    M = int(rng.integers(1, 1200 if big else 400))
+    N = int(rng.integers(1, 1500 if big else 500))
+    K = int(rng.integers(1, 6000 if big else 1500))
+    fa, fb = (int(rng.integers(0, 2)), int(rng.integers(0, 2)))
+    ma, mb = (int(rng.integers(0, 2)), int(rng.integers(0, 2)))
+    acc = int(rng.integers(0, 2))
+    out_dtype = torch.float32 if rng.integers(0, 2) else torch.bfloat16
+    A = _operand(rng, M if ma == api.MAJOR_K else K, K if ma == api.MAJOR_K else M, fa)
+    B = _operand(rng, N if mb == api.MAJOR_K else K, K if mb == api.MAJOR_K else N, fb)
+    sa, sb = float(2.0 ** rng.integers(-12, -2)), float(2.0 ** rng.integers(-6, 0))
+    esz = 4 if out_dtype == torch.float32 else 2
+    ldd = (N * esz + 15) // 16 * 16 // esz + (16 // esz) * int(rng.integers(0, 3))
+    D_full = torch.full((M + 1, ldd), 777.0, dtype=out_dtype, device=DEV)
+    D = D_full[:M, :N]
+    amax = torch.full((1,), -1.0, device=DEV)
+    api.fp8_gemm(A, fa, ma, B, fb, mb, D, torch.tensor([sa], device=DEV), torch.tensor([sb], device=DEV), amax, acc=acc)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    assert bool((D_full[M:, :] == 777.0).all()) and bool((D_full[:M, N:] == 777.0).all()), "wrote outside D"
+    ref, sabs = _reference(A, fa, ma, B, fb, mb, np.float64(np.float32(sa)) * np.float64(np.float32(sb)))
+    got = to_np_bits(D)
+    what = (M, N, K, fa, fb, ma, mb, acc, str(out_dtype))
+    if out_dtype == torch.float32:
+        ok, worst = check_gemm_f32(got, ref, sabs)
+        assert ok.all(), (what, worst, np.argwhere(~ok)[:4].tolist())
+    else:
+        ok, _ = check_gemm_bf16(got, ref, sabs, oracle.round_bf16_from_f64)
+        assert ok.all(), (what, np.argwhere(~ok)[:4].tolist())
+    assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(got.reshape(-1)), what
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_fp8_output_case(seed):
+    from tests._util import check_gemm_fp8out
+    rng = np.random.default_rng(7000 + seed)
+    M, N, K = int(rng.integers(1, 500)), int(rng.integers(1, 600)), int(rng.integers(1, 3000))
+    fa, fb, fd = int(rng.integers(0, 2)), int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    ma, mb, acc = int(rng.integers(0, 2)), int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    overflow = int(rng.integers(0, 2))
+    A = _operand(rng, M if ma == api.MAJOR_K else K, K if ma == api.MAJOR_K else M, fa)
+    B = _operand(rng, N if mb == api.MAJOR_K else K, K if mb == api.MAJOR_K else N, fb)
+    sa, sb = float(2.0 ** rng.integers(-12, -2)), float(2.0 ** rng.integers(-6, 0))
+    ref, sabs = _reference(A, fa, ma, B, fb, mb, np.float64(np.float32(sa)) * np.float64(np.float32(sb)))
+    # an output scale that puts the largest result near the top of the format, or (non-saturating runs) beyond it
+    peak = max(float(np.abs(ref).max()), 1e-30)
+    fmax = 448.0 if fd == oracle.E4M3 else 57344.0
+    scale_d = float(np.float32(fmax / peak * (4.0 if overflow == api.NOSAT and seed % 2 else 0.9)))
+    ldd = (N + 15) // 16 * 16 + 16 * int(rng.integers(0, 3))
+    D_full = torch.full((M + 1, ldd), 0xA5, dtype=torch.uint8, device=DEV)
+    D = D_full[:M, :N]
+    amax = torch.full((1,), -1.0, device=DEV)
+    dev = lambda v: torch.tensor([v], dtype=torch.float32, device=DEV)
+    api.fp8_gemm_fp8out(A, fa, ma, B, fb, mb, D, fd, dev(sa), dev(sb), dev(scale_d), amax, overflow, acc=acc)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    assert bool((D_full[M:, :] == 0xA5).all()) and bool((D_full[:M, N:] == 0xA5).all()), "wrote outside D"
+    enc = lambda y: oracle.quantize(y.reshape(-1), 1.0, fd, overflow).reshape(y.shape)
+    ok = check_gemm_fp8out(D.cpu().numpy(), ref, sabs, scale_d, enc)
+    assert ok.all(), ((M, N, K, fa, fb, fd, ma, mb, acc, overflow), np.argwhere(~ok)[:4].tolist())
+    lo = np.max(np.abs(ref) - 1e-5 * sabs) * (1 - 2.0 ** -22)
+    hi = np.max(np.abs(ref) + 1e-5 * sabs) * (1 + 2.0 ** -22)
+    assert lo <= float(amax.item()) <= hi
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_batched_and_splitk_case(seed):
+    rng = np.random.default_rng(5000 + seed)
+    fa, fb = int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    dev = lambda v: torch.tensor([v], dtype=torch.float32, device=DEV)
+    sa, sb = float(2.0 ** rng.integers(-12, -2)), float(2.0 ** rng.integers(-6, 0))
+    alpha = np.float64(np.float32(sa)) * np.float64(np.float32(sb))
+    if seed % 2 == 0:
+        # batched: heads side by side inside the rows of [S, H*d] operands
+        H, S, T, Dh = int(rng.integers(1, 6)), int(rng.integers(1, 300)), int(rng.integers(1, 300)), 16 * int(rng.integers(1, 9))
+        Qf = _operand(rng, S, H * Dh, fa)
+        Kf = _operand(rng, T, H * Dh, fb)
+        Q = Qf.as_strided((H, S, Dh), (Dh, Qf.stride(0), 1))
+        Kt = Kf.as_strided((H, T, Dh), (Dh, Kf.stride(0), 1))
+        ldd = (T + 3) // 4 * 4
+        D = torch.full((H, S + 1, ldd), 777.0, dtype=torch.float32, device=DEV)
+        amax = torch.full((1,), -1.0, device=DEV)
+        api.fp8_gemm_batched(Q, fa, api.MAJOR_K, Kt, fb, api.MAJOR_K, D[:, :S, :T], dev(sa), dev(sb), amax)
+        torch.cuda.synchronize()
+        assert api.fp8_async_status()[0] == 0
+        assert bool((D[:, S:, :] == 777.0).all()) and bool((D[:, :S, T:] == 777.0).all())
+        got = to_np_bits(D[:, :S, :T])
+        for h in range(H):
+            ref, sabs = _reference(Qf[:, h * Dh:(h + 1) * Dh], fa, api.MAJOR_K, Kf[:, h * Dh:(h + 1) * Dh], fb, api.MAJOR_K, alpha)
+            ok, worst = check_gemm_f32(got[h], ref, sabs)
+            assert ok.all(), (h, worst)
+        assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(got.reshape(-1))
+    else:
+        # split-K: few rows, long contraction
+        M, N, K = int(rng.integers(1, 260)), 4 * int(rng.integers(1, 300)), 256 * int(rng.integers(8, 80))
+        mb = int(rng.integers(0, 2))
+        A = _operand(rng, M, K, fa)
+        B = _operand(rng, N if mb == api.MAJOR_K else K, K if mb == api.MAJOR_K else N, fb)
+        splits, nbytes = api.fp8_gemm_splitk_workspace(M, N, K)
+        ws = torch.empty(max(nbytes // 4, 4), dtype=torch.float32, device=DEV)
+        out_dtype = torch.float32 if seed % 4 == 1 else torch.bfloat16
+        esz = 4 if out_dtype == torch.float32 else 2
+        ldd = (N * esz + 15) // 16 * 16 // esz
+        D_full = torch.full((M + 1, ldd), 777.0, dtype=out_dtype, device=DEV)
+        amax = torch.full((1,), -1.0, device=DEV)
+        api.fp8_gemm_splitk(A, fa, api.MAJOR_K, B, fb, mb, D_full[:M, :N], dev(sa), dev(sb), ws if nbytes else None, amax)
+        torch.cuda.synchronize()
+        assert api.fp8_async_status()[0] == 0
+        assert bool((D_full[M:, :] == 777.0).all()) and bool((D_full[:M, N:] == 777.0).all())
+        ref, sabs = _reference(A, fa, api.MAJOR_K, B, fb, mb, alpha)
+        got = to_np_bits(D_full[:M, :N])
+        if out_dtype == torch.float32:
+            ok, worst = check_gemm_f32(got, ref, sabs)
+        else:
+            ok, _ = check_gemm_bf16(got, ref, sabs, oracle.round_bf16_from_f64)
+        assert ok.all(), ((M, N, K, mb, splits), np.argwhere(~ok)[:4].tolist())
+        assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(got.reshape(-1))
