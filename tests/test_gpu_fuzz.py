@@ -163,3 +163,62 @@ def test_random_batched_and_splitk_case(seed):
             ok, _ = check_gemm_bf16(got, ref, sabs, oracle.round_bf16_from_f64)
         assert ok.all(), ((M, N, K, mb, splits), np.argwhere(~ok)[:4].tolist())
         assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(got.reshape(-1))
+
+
+@pytest.mark.parametrize("seed", range(64))
+def test_random_cast_case(seed):
+    """random length, pointer offsets, wide type, format, overflow mode and scale, special values sprinkled in:
+    quantize (+ amax), one-launch current scaling, dequantize and the simulated round trip against the oracle,
+    bit for bit, with guard elements around every output"""
+    from tests._util import same_with_nan
+    rng = np.random.default_rng(3000 + seed)
+    n = int(rng.integers(0, 1 << int(rng.integers(1, 20))))
+    wide = torch.float32 if rng.integers(0, 2) else torch.bfloat16
+    name = "f32" if wide == torch.float32 else "bf16"
+    fmt, overflow = int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    off_in, off_out = int(rng.integers(0, 16)), int(rng.integers(0, 16))
+    scale = float(np.float32(2.0 ** rng.uniform(-20, 20)))
+    vals = rng.standard_normal(n).astype(np.float32) * np.exp2(rng.uniform(-12, 12, size=n)).astype(np.float32)
+    if n:
+        specials = np.array([np.nan, -np.nan, np.inf, -np.inf, 0.0, -0.0, 448.0, 464.0, 465.0, 57344.0, 61440.0, 3e38, -3e38, 1e-40, 2.0 ** -9, 2.0 ** -17],
+                            dtype=np.float32)
+        where = rng.integers(0, n, size=max(1, n // 50))
+        vals[where] = specials[rng.integers(0, specials.size, size=where.size)]
+    base = torch.zeros(n + 32, dtype=wide, device=DEV)
+    x = base[off_in:off_in + n]
+    x.copy_(torch.from_numpy(vals).to(DEV).to(wide))
+    xh = to_np_bits(x)
+    dev = lambda v: torch.tensor([v], dtype=torch.float32, device=DEV)
+    # quantize + amax
+    out_full = torch.full((n + 48,), 0xA5, dtype=torch.uint8, device=DEV)
+    out = out_full[off_out:off_out + n]
+    amax = dev(-1.0)
+    api.fp8_quantize(x, fmt, dev(scale), out, overflow, amax)
+    want = oracle.quantize(xh, np.float32(scale), fmt, overflow)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), want), (n, name, fmt, overflow, off_in, off_out, scale)
+    assert bool((out_full[:off_out] == 0xA5).all()) and bool((out_full[off_out + n:] == 0xA5).all())
+    want_amax = oracle.amax_bits(xh) if n else 0
+    assert amax.cpu().numpy().view(np.uint32)[0] == want_amax
+    # one-launch current scaling
+    out_full.fill_(0xA5)
+    a2, s2, si2 = dev(-1.0), dev(-1.0), dev(-1.0)
+    api.fp8_quantize_current(x, fmt, out, a2, s2, si2, overflow)
+    ws, wsi = oracle.scale_from_amax(np.uint32(want_amax).view(np.float32), fmt)
+    torch.cuda.synchronize()
+    assert a2.cpu().numpy().view(np.uint32)[0] == want_amax and s2.item() == ws and si2.item() == wsi
+    want2 = oracle.quantize(xh, ws, fmt, overflow)
+    assert np.array_equal(out.cpu().numpy(), want2)
+    assert bool((out_full[:off_out] == 0xA5).all()) and bool((out_full[off_out + n:] == 0xA5).all())
+    # dequantize of those codes, and the simulated round trip
+    back_full = torch.full((n + 48,), 7.0, dtype=wide, device=DEV)
+    back = back_full[off_out:off_out + n]
+    api.fp8_dequantize(out, fmt, si2, back)
+    torch.cuda.synchronize()
+    assert same_with_nan(to_np_bits(back), oracle.dequantize(want2, wsi, fmt, name), name).all()
+    assert bool((back_full[:off_out] == 7.0).all()) and bool((back_full[off_out + n:] == 7.0).all())
+    back_full.fill_(7.0)
+    api.fp8_fake_quantize(x, fmt, s2, si2, back, overflow)
+    torch.cuda.synchronize()
+    assert same_with_nan(to_np_bits(back), oracle.fake_quantize(xh, ws, wsi, fmt, overflow), name).all()
+    assert bool((back_full[:off_out] == 7.0).all()) and bool((back_full[off_out + n:] == 7.0).all())
