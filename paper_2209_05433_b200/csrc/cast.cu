@@ -1,10 +1,12 @@
 // amax, scale selection, quantize (wide -> FP8) and dequantize (FP8 -> wide):
 // the memory-bound half of the FP8 hot path (Section 2 of the paper).
 //
-// All four tensor kernels are persistent grid-stride loops over 16-byte items
-// with several independent 128-bit loads in flight per thread; every warp-level
-// load and store instruction covers one contiguous span.  HBM traffic is the
-// algorithmic minimum (each input byte read once, each output byte written once).
+// The flat tensor kernels (amax, quantize, dequantize, the simulated round trip and the one-launch
+// current scaling) are persistent grid-stride loops over 16-byte items with several independent
+// 128-bit loads in flight per thread; every warp-level load and store instruction covers one
+// contiguous span.  HBM traffic is the algorithmic minimum (each input byte read once per pass, each
+// output byte written once).  The 2-D kernels (per-row / per-column scales, quantize with a transposed
+// copy) follow the same rules with shapes of their own, described at each kernel.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
