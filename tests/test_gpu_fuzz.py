@@ -222,3 +222,54 @@ def test_random_cast_case(seed):
     torch.cuda.synchronize()
     assert same_with_nan(to_np_bits(back), oracle.fake_quantize(xh, ws, wsi, fmt, overflow), name).all()
     assert bool((back_full[:off_out] == 7.0).all()) and bool((back_full[off_out + n:] == 7.0).all())
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_channel_and_transpose_case(seed):
+    """random 2-D shapes, pitches and base offsets through the per-channel kernels (both axes) and the transposing
+    quantizer, with special values sprinkled in; everything bit-exact against the oracle"""
+    rng = np.random.default_rng(1000 + seed)
+    rows, cols = int(rng.integers(1, 700)), int(rng.integers(1, 900))
+    if seed % 3 == 0:                                       # shapes the vector paths accept
+        rows, cols = 4 * int(rng.integers(1, 200)), 8 * int(rng.integers(1, 150))
+    wide = torch.float32 if rng.integers(0, 2) else torch.bfloat16
+    fmt, overflow, axis = int(rng.integers(0, 2)), int(rng.integers(0, 2)), int(rng.integers(0, 2))
+    pitch = cols + (8 * int(rng.integers(0, 3)) if seed % 3 == 0 else int(rng.integers(0, 9)))
+    off = 0 if seed % 3 == 0 else int(rng.integers(0, 8))
+    vals = rng.standard_normal(rows * pitch).astype(np.float32) * np.exp2(rng.uniform(-8, 8, size=rows * pitch)).astype(np.float32)
+    specials = np.array([np.nan, -np.nan, np.inf, -np.inf, 0.0, -0.0, 448.0, 465.0, 61440.0, 3e38, 1e-40], dtype=np.float32)
+    where = rng.integers(0, vals.size, size=max(1, vals.size // 200))
+    vals[where] = specials[rng.integers(0, specials.size, size=where.size)]
+    base = torch.zeros(rows * pitch + 16, dtype=wide, device=DEV)
+    base[off:off + rows * pitch] = torch.from_numpy(vals).to(DEV).to(wide)
+    x = base[off:off + rows * pitch].view(rows, pitch)[:, :cols]
+    xh = to_np_bits(x)
+    # per-channel amax -> scales -> quantize
+    nch = cols if axis == 0 else rows
+    am = torch.full((nch,), -1.0, device=DEV)
+    sv, siv = torch.empty(nch, device=DEV), torch.empty(nch, device=DEV)
+    api.fp8_amax_channels(x, axis, am)
+    api.fp8_scales_from_amax(am, fmt, sv, siv)
+    opitch = cols + int(rng.integers(0, 3)) * (8 if seed % 3 == 0 else 1)
+    q_full = torch.full((rows + 1, opitch), 0xA5, dtype=torch.uint8, device=DEV)
+    api.fp8_quantize_channels(x, axis, fmt, sv, q_full[:rows, :cols], overflow)
+    torch.cuda.synchronize()
+    want_am = oracle.amax_channels(xh, axis)
+    assert np.array_equal(am.cpu().numpy().view(np.uint32), want_am.view(np.uint32)), (rows, cols, axis, str(wide))
+    ws, wsi = oracle.scales_from_amax(want_am, fmt)
+    assert np.array_equal(sv.cpu().numpy(), ws) and np.array_equal(siv.cpu().numpy(), wsi)
+    assert np.array_equal(q_full[:rows, :cols].cpu().numpy(), oracle.quantize_channels(xh, ws, axis, fmt, overflow))
+    assert bool((q_full[rows:, :] == 0xA5).all()) and bool((q_full[:rows, cols:] == 0xA5).all())
+    # quantize + transposed copy with one scale
+    scale = float(np.float32(2.0 ** rng.uniform(-6, 6)))
+    tpitch = rows + int(rng.integers(0, 3)) * (4 if seed % 3 == 0 else 1)
+    q_full.fill_(0xA5)
+    t_full = torch.full((cols + 1, tpitch), 0xA5, dtype=torch.uint8, device=DEV)
+    amax = torch.full((1,), -1.0, device=DEV)
+    api.fp8_quantize_transpose(x, fmt, torch.tensor([scale], device=DEV), q_full[:rows, :cols], t_full[:cols, :rows], amax, overflow)
+    torch.cuda.synchronize()
+    want = oracle.quantize(xh.reshape(-1), np.float32(scale), fmt, overflow).reshape(rows, cols)
+    assert np.array_equal(q_full[:rows, :cols].cpu().numpy(), want) and np.array_equal(t_full[:cols, :rows].cpu().numpy(), want.T)
+    assert bool((q_full[rows:, :] == 0xA5).all()) and bool((q_full[:rows, cols:] == 0xA5).all())
+    assert bool((t_full[cols:, :] == 0xA5).all()) and bool((t_full[:cols, rows:] == 0xA5).all())
+    assert amax.cpu().numpy().view(np.uint32)[0] == oracle.amax_bits(xh.reshape(-1))
