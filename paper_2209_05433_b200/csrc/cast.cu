@@ -54,6 +54,25 @@ constexpr int kWideBF16 = 1;
 #endif
 constexpr int kThreads = FP8_CAST_THREADS;
 
+// Input loads of the streaming kernels: read-only path without L1 allocation.  Plain loads (FP8_PLAIN_LOADS) were
+// measured too: faster on tensors far larger than L2 (amax +4 %, quantize +2.5 %, binary32-input quantize +7 %) but
+// slower whenever part of the tensor sits in L2 (2^24 elements: amax 2950 -> 2194 GB/s; per-column kernels -6..-15 %)
+// and 2 % slower for the casts inside the benchmark step, so they are not the default.
+__device__ __forceinline__ uint4 ld_in_v4(const void* p) {
+#ifdef FP8_PLAIN_LOADS
+    return *reinterpret_cast<const uint4*>(p);
+#else
+    return ld_nc_v4(p);
+#endif
+}
+__device__ __forceinline__ uint2 ld_in_v2(const void* p) {
+#ifdef FP8_PLAIN_LOADS
+    return *reinterpret_cast<const uint2*>(p);
+#else
+    return ld_nc_v2(p);
+#endif
+}
+
 // Output stores: written once, never re-read by the same kernel.
 __device__ __forceinline__ void st_out(uint2* p, uint2 v) {
 #ifdef FP8_STORE_CS
@@ -199,14 +218,14 @@ __global__ void __launch_bounds__(kThreads) k_amax(const void* __restrict__ x, s
         uint4 v[UNROLL];
         if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
+            for (int u = 0; u < UNROLL; ++u) v[u] = ld_in_v4(xv + base + (size_t)u * kThreads);
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) m = fold_abs_max<WIDE>(m, v[u]);
         } else {
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const size_t i = base + (size_t)u * kThreads;
-                if (i < n_items) m = fold_abs_max<WIDE>(m, ld_nc_v4(xv + i));
+                if (i < n_items) m = fold_abs_max<WIDE>(m, ld_in_v4(xv + i));
             }
         }
     }
@@ -241,14 +260,14 @@ k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale
         if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
             uint4 v[UNROLL];
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
+            for (int u = 0; u < UNROLL; ++u) v[u] = ld_in_v4(xv + base + (size_t)u * kThreads);
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) emit(base + (size_t)u * kThreads, v[u]);
         } else {
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const size_t i = base + (size_t)u * kThreads;
-                if (i < n_items) emit(i, ld_nc_v4(xv + i));
+                if (i < n_items) emit(i, ld_in_v4(xv + i));
             }
         }
     }
@@ -297,7 +316,7 @@ k_dequantize(const uint8_t* __restrict__ c, size_t n, const float* __restrict__ 
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const size_t i = base + (size_t)u * kThreads;
-                if (full || i < n_items) v[u] = ld_nc_v2(c + i * 8);
+                if (full || i < n_items) v[u] = ld_in_v2(c + i * 8);
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
@@ -392,6 +411,34 @@ __device__ unsigned int g_cast_latch[2] = {0u, 0u};
 constexpr unsigned int kWaitGridBarrier = 16u;
 constexpr long long kGridWaitLimitCycles = 4000000000ll;       // about 2 s of SM clocks
 
+// One-launch current scaling: megabytes of the end of x asked to stay in L2 between the passes, for tensors
+// larger than FP8_CURRENT_KEEP_FROM_MB (smaller ones are left to the default replacement: they mostly fit).
+// Measured together with plain second-pass loads: 106.2 -> 96.9 us on [8192 x 16384] bf16, 419 -> 399 us on 2^29
+// elements; [4096 x 16384] 52.5 -> 47.8 us and [8192 x 4096] 20.2 -> 19.2 us from the plain loads alone.
+#ifndef FP8_CURRENT_KEEP_MB
+#define FP8_CURRENT_KEEP_MB 96
+#endif
+#ifndef FP8_CURRENT_KEEP_FROM_MB
+#define FP8_CURRENT_KEEP_FROM_MB 160
+#endif
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint4 ld_v4_policy(const void* ptr, uint64_t policy) {
+    uint4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr), "l"(policy));
+    return v;
+}
+
+
 // Current scaling in ONE launch: amax of x, scale = fmax / amax, quantize with that scale.
 // All CTAs are co-resident (cooperative launch).  ws[0] = running amax bits, ws[1] = arrivals at the
 // grid barrier, ws[2] = departures; the three words are zero on entry and the last CTA to leave puts
@@ -411,13 +458,22 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
     const size_t tail = n - n_items * EPI;
 
     // ---- pass 1: amax
+    // a large tensor: its last FP8_CURRENT_KEEP_MB megabytes are asked to stay in L2 for the second pass (which
+    // starts there), the rest to leave first; a small one: default replacement
+    const bool large = n_chunks * per_chunk * 16 > ((size_t)FP8_CURRENT_KEEP_FROM_MB << 20);
+    const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
+    const size_t keep_chunks = ((size_t)FP8_CURRENT_KEEP_MB << 20) / (per_chunk * 16);
+    const size_t keep_from = n_chunks > keep_chunks ? n_chunks - keep_chunks : 0;
     uint32_t m = 0;
     for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
         const size_t base = chunk * per_chunk + threadIdx.x;
         if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
             uint4 v[UNROLL];
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) v[u] = *(xv + base + (size_t)u * kThreads);   // default caching: kept in L2 for pass 2
+            for (int u = 0; u < UNROLL; ++u) {
+                if (large) v[u] = ld_v4_policy(xv + base + (size_t)u * kThreads, chunk >= keep_from ? pol_keep : pol_stream);
+                else       v[u] = *(xv + base + (size_t)u * kThreads);
+            }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) m = fold_abs_max<WIDE>(m, v[u]);
         } else {
@@ -478,7 +534,8 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
             if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
                 uint4 v[UNROLL];
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
+                // plain loads: the read-only no-allocate path measured 3-9 % slower on this re-read
+                for (int u = 0; u < UNROLL; ++u) v[u] = *(xv + base + (size_t)u * kThreads);
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) {
                     const size_t i = base + (size_t)u * kThreads;
@@ -490,7 +547,7 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
                 for (int u = 0; u < UNROLL; ++u) {
                     const size_t i = base + (size_t)u * kThreads;
                     if (i < n_items) {
-                        const uint4 v = ld_nc_v4(xv + i);
+                        const uint4 v = ld_in_v4(xv + i);
                         if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out) + i, quantize_item_bf16<FMT, NOSAT>(v, scale));
                         else                   st_out(reinterpret_cast<uint32_t*>(out) + i, quantize_item_f32<FMT, NOSAT>(v, scale));
                     }
@@ -646,11 +703,11 @@ k_amax_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, 
         for (; r + (kColsUnroll - 1) * kColsTy < r1; r += kColsUnroll * kColsTy) {
             uint4 v[kColsUnroll];
 #pragma unroll
-            for (int u = 0; u < kColsUnroll; ++u) v[u] = ld_nc_v4(base + (r + u * kColsTy) * ld * ESZ);
+            for (int u = 0; u < kColsUnroll; ++u) v[u] = ld_in_v4(base + (r + u * kColsTy) * ld * ESZ);
 #pragma unroll
             for (int u = 0; u < kColsUnroll; ++u) fold(v[u]);
         }
-        for (; r < r1; r += kColsTy) fold(ld_nc_v4(base + r * ld * ESZ));
+        for (; r < r1; r += kColsTy) fold(ld_in_v4(base + r * ld * ESZ));
     }
     part[ty][tx] = m;
     __syncthreads();
@@ -696,11 +753,11 @@ k_amax_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t ld, 
         for (; i + 32 * (kRowsAmaxUnroll - 1) < end; i += 32 * kRowsAmaxUnroll) {
             uint4 v[kRowsAmaxUnroll];
 #pragma unroll
-            for (int k = 0; k < kRowsAmaxUnroll; ++k) v[k] = ld_nc_v4(row + (i + 32 * k) * 16);
+            for (int k = 0; k < kRowsAmaxUnroll; ++k) v[k] = ld_in_v4(row + (i + 32 * k) * 16);
 #pragma unroll
             for (int k = 0; k < kRowsAmaxUnroll; ++k) m = fold_abs_max<WIDE>(m, v[k]);
         }
-        for (; i < end; i += 32) m = fold_abs_max<WIDE>(m, ld_nc_v4(row + i * 16));
+        for (; i < end; i += 32) m = fold_abs_max<WIDE>(m, ld_in_v4(row + i * 16));
         m = finish_abs_max<WIDE>(m);
         if (seg == segs - 1)                                          // ragged tail of the row
             for (int64_t c = n_items * EPI + lane; c < cols; c += 32) m = max(m, canonical_nan_bits(scalar_abs_bits<WIDE>(row, c)));
@@ -790,11 +847,11 @@ k_quantize_cols(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t 
     for (; r + 3 * kColsTy < r1; r += 4 * kColsTy) {
         uint4 v[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = ld_nc_v4(base + (r + u * kColsTy) * ld * ESZ);
+        for (int u = 0; u < 4; ++u) v[u] = ld_in_v4(base + (r + u * kColsTy) * ld * ESZ);
 #pragma unroll
         for (int u = 0; u < 4; ++u) emit(r + u * kColsTy, v[u]);
     }
-    for (; r < r1; r += kColsTy) emit(r, ld_nc_v4(base + r * ld * ESZ));
+    for (; r < r1; r += kColsTy) emit(r, ld_in_v4(base + r * ld * ESZ));
 }
 
 // AXIS 1, vector path: a warp per (row, segment) unit as in k_amax_rows, the row's scale in a register.
@@ -821,11 +878,11 @@ k_quantize_rows(const void* __restrict__ x, int64_t rows, int64_t cols, int64_t 
         if (i0 + 32 * (kRowsUnroll - 1) < n_items) {
             uint4 v[kRowsUnroll];
 #pragma unroll
-            for (int k = 0; k < kRowsUnroll; ++k) v[k] = ld_nc_v4(row + (i0 + 32 * k) * 16);
+            for (int k = 0; k < kRowsUnroll; ++k) v[k] = ld_in_v4(row + (i0 + 32 * k) * 16);
 #pragma unroll
             for (int k = 0; k < kRowsUnroll; ++k) emit(orow, i0 + 32 * k, v[k], s);
         } else {
-            for (int64_t i = i0; i < n_items; i += 32) emit(orow, i, ld_nc_v4(row + i * 16), s);
+            for (int64_t i = i0; i < n_items; i += 32) emit(orow, i, ld_in_v4(row + i * 16), s);
         }
         if (seg == segs - 1) {
             for (int64_t c = n_items * EPI + lane; c < cols; c += 32) {
@@ -942,7 +999,7 @@ k_quantize_transpose(const void* __restrict__ x, int64_t rows, int64_t cols, int
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             v[s][i] = make_uint4(0u, 0u, 0u, 0u);
-            if (col_ok && r + i < rows) v[s][i] = ld_nc_v4(xb + ((r + i) * ldx + c) * ESZ);
+            if (col_ok && r + i < rows) v[s][i] = ld_in_v4(xb + ((r + i) * ldx + c) * ESZ);
         }
     }
 #pragma unroll
