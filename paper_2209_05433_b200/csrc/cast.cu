@@ -421,6 +421,9 @@ constexpr long long kGridWaitLimitCycles = 4000000000ll;       // about 2 s of S
 #ifndef FP8_CURRENT_KEEP_FROM_MB
 #define FP8_CURRENT_KEEP_FROM_MB 160
 #endif
+#ifndef FP8_CURRENT_PLAIN_REREAD
+#define FP8_CURRENT_PLAIN_REREAD 1
+#endif
 __device__ __forceinline__ uint64_t l2_policy_evict_last() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
@@ -460,7 +463,7 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
     // ---- pass 1: amax
     // a large tensor: its last FP8_CURRENT_KEEP_MB megabytes are asked to stay in L2 for the second pass (which
     // starts there), the rest to leave first; a small one: default replacement
-    const bool large = n_chunks * per_chunk * 16 > ((size_t)FP8_CURRENT_KEEP_FROM_MB << 20);
+    const bool large = FP8_CURRENT_KEEP_MB > 0 && n_chunks * per_chunk * 16 > ((size_t)FP8_CURRENT_KEEP_FROM_MB << 20);
     const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
     const size_t keep_chunks = ((size_t)FP8_CURRENT_KEEP_MB << 20) / (per_chunk * 16);
     const size_t keep_from = n_chunks > keep_chunks ? n_chunks - keep_chunks : 0;
@@ -534,8 +537,11 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
             if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
                 uint4 v[UNROLL];
 #pragma unroll
-                // plain loads: the read-only no-allocate path measured 3-9 % slower on this re-read
+#if FP8_CURRENT_PLAIN_REREAD
                 for (int u = 0; u < UNROLL; ++u) v[u] = *(xv + base + (size_t)u * kThreads);
+#else
+                for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
+#endif
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) {
                     const size_t i = base + (size_t)u * kThreads;
