@@ -24,7 +24,8 @@ def _scalar():
 
 
 def _cast(x, fmt, rng):
-    """two-pass current scaling through the library; verified against the oracle; returns (codes, scale_inv, host codes)"""
+    """current scaling through the library, as three calls and as the one launch the benchmark times; verified
+    against the oracle; returns (codes, scale_inv, host codes, oracle's scale_inv)"""
     n = x.numel()
     a, s, si = _scalar(), _scalar(), _scalar()
     codes = torch.empty(n, dtype=torch.uint8, device=DEV)
@@ -41,6 +42,14 @@ def _cast(x, fmt, rng):
     for lo, hi in blocks:
         want = oracle.quantize(x_host[lo:hi], ws, fmt, threads=THREADS)
         assert np.array_equal(codes_host[lo:hi], want), (lo, hi)
+    # the one-launch form the benchmark step uses: same amax, scales and codes, everywhere
+    a1, s1, si1 = _scalar(), _scalar(), _scalar()
+    codes1 = torch.empty(n, dtype=torch.uint8, device=DEV)
+    api.fp8_quantize_current(x.view(-1), fmt, codes1, a1, s1, si1)
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    assert a1.item() == a.item() and s1.item() == ws and si1.item() == wsi
+    assert torch.equal(codes1, codes)
     return codes, si, codes_host, wsi
 
 
