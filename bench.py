@@ -1,25 +1,30 @@
 #!/usr/bin/env python
 """Benchmark of the FP8 hot path on B200.
 
-One "step" is one pass of the whole hot path over one synthetic batch of a
-transformer linear layer (hidden 4096 -> 16384, 8192 tokens): for each of the
-activations X, weights W (E4M3) and output gradients dY (E5M2) the two-pass
-current scaling  amax -> scale -> quantize, one dequantize (the FP8 -> bf16
-round trip), then the three FP8 GEMMs with fp32 accumulation and bf16 output
-with epilogue amax: forward Y = X.W, dgrad dX = dY.W^T, wgrad dW = X^T.dY.
+One "step" is one pass of the whole hot path over one synthetic batch of the largest workload,
+the 175B-class FFN layer (hidden 12288 -> 49152, 8192 tokens): for each of the activations X,
+weights W (E4M3) and output gradients dY (E5M2) the two-pass current scaling
+amax -> scale -> quantize, one dequantize (the FP8 -> bf16 round trip), then the FP8 GEMMs with
+fp32 accumulation and bf16 output with epilogue amax: forward Y = X.W and dgrad dX = dY.W^T.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-Prints ONE JSON line.  `value` is whole-job TFLOP/s: GEMM flops of all ranks
-divided by the max-over-ranks device time of the K steps, casts included.
-`--impl reference` times the CPU oracle (the slow checker under oracle/) on a
-bounded sample of the same step instead.
+Prints ONE JSON line.  `value` is whole-job TFLOP/s: GEMM flops of all ranks divided by the
+max-over-ranks device time of the K steps, casts included.  With --gpus N > 1 and no torchrun
+environment the script starts its N ranks itself (one process per GPU).  `--impl reference`
+times the CPU oracle (the slow checker under oracle/) on a bounded sample of the same step.
+
+Two regimes are reported and labelled: the K timed steps (a fraction of a second: the GPU is
+still at boost clocks, "burst") and a loop of whole steps lasting at least two seconds under
+the power cap ("sustained").  Roofline fractions divide burst figures by the burst peak and
+sustained figures by the sustained peak.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -32,15 +37,22 @@ if ROOT not in sys.path:
 
 METRIC = "fp8_linear_step_gemm_tflops"
 UNIT = "TFLOP/s"
-WORKLOAD = ("transformer linear layer fwd+bwd, hidden 4096->16384, 8192 tokens: amax+scale+quantize of X,W (E4M3) and dY (E5M2), "
-            "one dequantize, fprop/dgrad/wgrad FP8 GEMMs, bf16 out + epilogue amax")
-TOKENS, D_IN, D_OUT, W_SIGMA = 8192, 4096, 16384, 0.02
-# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (same workload):
-# forward GEMM 168.5 MB + 225.5 MB; one-launch conversion, mean of the X, W and dY launches.
-NCU_TRAFFIC_GEMM_BYTES = 3.94e8
-NCU_TRAFFIC_QUANTIZE_CURRENT_BYTES = 2.68e8
 NOMINAL_FP8_TFLOPS = 4500.0
 NOMINAL_HBM_GBS = 8000.0
+FP8_MACS_PER_SM_PER_CLOCK = 8192           # dense 8-bit multiply-adds one SM's tensor pipe retires per clock
+
+# (tokens, d_in, d_out, sigma of the weights, seed, GEMM passes) of the layer workloads
+LAYERS = {
+    "hidden4096": dict(tokens=8192, d_in=4096, d_out=16384, w_sigma=0.02, seed=3, passes=("fprop", "dgrad", "wgrad")),
+    "hidden12288": dict(tokens=8192, d_in=12288, d_out=49152, w_sigma=0.006, seed=5, passes=("fprop", "dgrad")),
+}
+HEADLINE = "hidden12288"
+
+
+def workload_text(layer):
+    L = LAYERS[layer]
+    return ("transformer FFN linear layer, hidden %d->%d, %d tokens: amax+scale+quantize of X, W (E4M3) and dY (E5M2), "
+            "one dequantize, %s FP8 GEMMs, bf16 out + epilogue amax" % (L["d_in"], L["d_out"], L["tokens"], "/".join(L["passes"])))
 
 
 def peaks():
@@ -53,6 +65,21 @@ def peaks():
                     bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
     except Exception:
         return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def ncu_traffic():
+    """DRAM bytes per launch (read + write) of the profiled kernels, from the table the ncu summaries keep:
+    lines of `name  bytes  ...`; a name missing from the table gives None."""
+    table = {}
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 2 and not line.startswith("#"):
+                    table[parts[0]] = float(parts[1])
+    except OSError:
+        pass
+    return table
 
 
 # ----------------------------------------------------------------------------
@@ -107,7 +134,7 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
         busy = [c for c, p in zip(sm, power) if p >= 0.5 * max(power)] or sm
         return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "power_w_max": max(power),
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "samples_under_load": len(busy), "reasons": sorted(reasons)}
 
 
 # ----------------------------------------------------------------------------
@@ -117,63 +144,56 @@ class ClockSampler:
 class LinearStep:
     """Buffers and call sequence of one step.  Everything the step computes runs in the library's kernels."""
 
-    def __init__(self, torch, api, synth, device, seed, tokens=TOKENS, d_in=D_IN, d_out=D_OUT, fused_cast=True):
-        self.torch, self.api = torch, api
-        self.fused_cast = fused_cast
-        self.T, self.I, self.O = tokens, d_in, d_out
-        dev = device
+    def __init__(self, torch, api, synth, device, layer, seed_offset=0):
+        L = LAYERS[layer]
+        self.torch, self.api, self.layer = torch, api, layer
+        self.T, self.I, self.O, self.passes = L["tokens"], L["d_in"], L["d_out"], L["passes"]
+        T, I, O, seed = self.T, self.I, self.O, L["seed"] + seed_offset
         bf, u8, f32 = torch.bfloat16, torch.uint8, torch.float32
-        self.X = synth.activations(tokens * d_in, seed, dtype=bf, device=dev).view(tokens, d_in)
-        self.W = synth.weights(d_in * d_out, seed, W_SIGMA, dtype=bf, device=dev).view(d_in, d_out)
-        self.dY = synth.gradients(tokens * d_out, seed + 1, dtype=bf, device=dev).view(tokens, d_out)
-        self.Xq = torch.empty(tokens, d_in, dtype=u8, device=dev)
-        self.Wq = torch.empty(d_in, d_out, dtype=u8, device=dev)
-        self.dYq = torch.empty(tokens, d_out, dtype=u8, device=dev)
-        self.Xhat = torch.empty(tokens, d_in, dtype=bf, device=dev)
-        self.Y = torch.empty(tokens, d_out, dtype=bf, device=dev)
-        self.dX = torch.empty(tokens, d_in, dtype=bf, device=dev)
-        self.dW = torch.empty(d_in, d_out, dtype=bf, device=dev)
-        self.scal = torch.zeros(16, dtype=f32, device=dev)      # amax / scale / scale_inv per tensor, GEMM amaxes
+        self.X = synth.activations(T * I, seed, dtype=bf, device=device).view(T, I)
+        self.W = synth.weights(I * O, seed, L["w_sigma"], dtype=bf, device=device).view(I, O)
+        self.dY = synth.gradients(T * O, seed + (1 if layer == "hidden4096" else 0), dtype=bf, device=device).view(T, O)
+        self.Xq = torch.empty(T, I, dtype=u8, device=device)
+        self.Wq = torch.empty(I, O, dtype=u8, device=device)
+        self.dYq = torch.empty(T, O, dtype=u8, device=device)
+        self.Xhat = torch.empty(T, I, dtype=bf, device=device)
+        self.Y = torch.empty(T, O, dtype=bf, device=device) if "fprop" in self.passes else None
+        self.dX = torch.empty(T, I, dtype=bf, device=device) if "dgrad" in self.passes else None
+        self.dW = torch.empty(I, O, dtype=bf, device=device) if "wgrad" in self.passes else None
+        self.scal = torch.zeros(16, dtype=f32, device=device)      # amax / scale / scale_inv per tensor, GEMM amaxes
         s = [self.scal[i:i + 1] for i in range(16)]
         self.ax, self.sx, self.six, self.aw, self.sw, self.siw, self.ag, self.sg, self.sig = s[:9]
         self.ay, self.adx, self.adw = s[9:12]
-        self.gemm_flops = 3 * 2.0 * tokens * d_in * d_out
+        self.flops_per_gemm = 2.0 * T * I * O
+        self.gemm_flops = len(self.passes) * self.flops_per_gemm
         # algorithmic HBM bytes of the cast part: two-pass (read, read, write) = 5 B per bf16 element; dequantize 3 B
-        n_cast = tokens * d_in + d_in * d_out + tokens * d_out
-        self.cast_bytes = 5.0 * n_cast + 3.0 * tokens * d_in
+        self.n_cast = T * I + I * O + T * O
+        self.cast_bytes = 5.0 * self.n_cast + 3.0 * T * I
+        self.inputs = (self.X, self.W, self.dY)
+        self.outputs = tuple(t for t in (self.Y, self.dX, self.dW) if t is not None)
 
     def calls(self):
         """(label, thunk) for every library call of one step, in order"""
         a = self.api
         E4, E5, KM, MN = a.E4M3, a.E5M2, a.MAJOR_K, a.MAJOR_MN
-        if self.fused_cast:
-            casts = [
-                # amax -> scale -> quantize of one tensor in one cooperative launch
-                ("quantize_current", lambda: a.fp8_quantize_current(self.X, E4, self.Xq, self.ax, self.sx, self.six)),
-                ("quantize_current", lambda: a.fp8_quantize_current(self.W, E4, self.Wq, self.aw, self.sw, self.siw)),
-                ("quantize_current", lambda: a.fp8_quantize_current(self.dY, E5, self.dYq, self.ag, self.sg, self.sig)),
-            ]
-        else:
-            casts = [
-                ("amax", lambda: a.fp8_amax(self.X, self.ax)),
-                ("scale", lambda: a.fp8_scale_from_amax(self.ax, E4, self.sx, self.six)),
-                ("quantize", lambda: a.fp8_quantize(self.X, E4, self.sx, self.Xq)),
-                ("amax", lambda: a.fp8_amax(self.W, self.aw)),
-                ("scale", lambda: a.fp8_scale_from_amax(self.aw, E4, self.sw, self.siw)),
-                ("quantize", lambda: a.fp8_quantize(self.W, E4, self.sw, self.Wq)),
-                ("amax", lambda: a.fp8_amax(self.dY, self.ag)),
-                ("scale", lambda: a.fp8_scale_from_amax(self.ag, E5, self.sg, self.sig)),
-                ("quantize", lambda: a.fp8_quantize(self.dY, E5, self.sg, self.dYq)),
-            ]
-        return casts + [
+        calls = [
+            # amax -> scale -> quantize of one tensor in one cooperative launch
+            ("quantize_current_X", lambda: a.fp8_quantize_current(self.X, E4, self.Xq, self.ax, self.sx, self.six)),
+            ("quantize_current_W", lambda: a.fp8_quantize_current(self.W, E4, self.Wq, self.aw, self.sw, self.siw)),
+            ("quantize_current_dY", lambda: a.fp8_quantize_current(self.dY, E5, self.dYq, self.ag, self.sg, self.sig)),
             ("dequantize", lambda: a.fp8_dequantize(self.Xq, E4, self.six, self.Xhat)),
-            # forward: Y[T,O] = X[T,I] . W[I,O]   (W stored with the output index contiguous)
-            ("gemm_fprop", lambda: a.fp8_gemm(self.Xq, E4, KM, self.Wq, E4, MN, self.Y, self.six, self.siw, self.ay)),
-            # dgrad: dX[T,I] = dY[T,O] . W^T      (W stored [I,O] is the [N,K] layout here)
-            ("gemm_dgrad", lambda: a.fp8_gemm(self.dYq, E5, KM, self.Wq, E4, KM, self.dX, self.sig, self.siw, self.adx)),
-            # wgrad: dW[I,O] = X^T . dY           (both operands stored with the contraction index outermost)
-            ("gemm_wgrad", lambda: a.fp8_gemm(self.Xq, E4, MN, self.dYq, E5, MN, self.dW, self.six, self.sig, self.adw)),
         ]
+        if "fprop" in self.passes:      # Y[T,O] = X[T,I] . W[I,O]   (W stored with the output index contiguous)
+            calls.append(("gemm_fprop", lambda: a.fp8_gemm(self.Xq, E4, KM, self.Wq, E4, MN, self.Y, self.six, self.siw, self.ay)))
+        if "dgrad" in self.passes:      # dX[T,I] = dY[T,O] . W^T      (W stored [I,O] is the [N,K] layout here)
+            calls.append(("gemm_dgrad", lambda: a.fp8_gemm(self.dYq, E5, KM, self.Wq, E4, KM, self.dX, self.sig, self.siw, self.adx)))
+        if "wgrad" in self.passes:      # dW[I,O] = X^T . dY           (both operands stored with the contraction index outermost)
+            calls.append(("gemm_wgrad", lambda: a.fp8_gemm(self.Xq, E4, MN, self.dYq, E5, MN, self.dW, self.six, self.sig, self.adw)))
+        return calls
+
+    def cast_elements(self, label):
+        return {"quantize_current_X": self.T * self.I, "quantize_current_W": self.I * self.O,
+                "quantize_current_dY": self.T * self.O, "dequantize": self.T * self.I}[label]
 
     def run(self, only=None):
         for label, f in self.calls():
@@ -195,44 +215,31 @@ class LinearStep:
         events.append(row)
 
 
-def bench_cast_sweep(torch, api, synth, device, log2n, iters=20):
-    """config-2 style bandwidth point: bf16 tensors of 2^log2n elements; single-pass quantize+amax, amax, dequantize.
-    Calls alternate between two distinct tensors, so that no call finds in L2 what the previous one left there
-    (the two-pass kernel ends its second pass where its first pass starts)."""
-    n = 1 << log2n
-    xs = [synth.normal_laplace_mixture(n, 1 + k, synth.T_ID, device=device) for k in range(2)]
-    codes = [torch.empty(n, dtype=torch.uint8, device=device) for _ in range(2)]
-    backs = [torch.empty(n, dtype=torch.bfloat16, device=device) for _ in range(2)]
-    sc = torch.tensor([3.0, 1.0 / 3.0, 0.0], dtype=torch.float32, device=device)
-    s, si, a = sc[0:1], sc[1:2], sc[2:3]
-    sc2 = torch.zeros(2, dtype=torch.float32, device=device)
-    s2, si2 = sc2[0:1], sc2[1:2]
-    out = {}
-    cases = {
-        "quantize_e4m3_with_amax": (lambda i: api.fp8_quantize(xs[i], api.E4M3, s, codes[i], api.SATURATE, a), 3.0 * n),
-        "quantize_e5m2_with_amax": (lambda i: api.fp8_quantize(xs[i], api.E5M2, s, codes[i], api.SATURATE, a), 3.0 * n),
-        "amax": (lambda i: api.fp8_amax(xs[i], a), 2.0 * n),
-        "quantize_current_e4m3": (lambda i: api.fp8_quantize_current(xs[i], api.E4M3, codes[i], a, s2, si2), 5.0 * n),
-        "dequantize_e4m3": (lambda i: api.fp8_dequantize(codes[i], api.E4M3, si, backs[i]), 3.0 * n),
-        "fake_quantize_e4m3": (lambda i: api.fp8_fake_quantize(xs[i], api.E4M3, s, si, backs[i]), 4.0 * n),
-    }
-    for name, (fn, nbytes) in cases.items():
-        for k in range(4):
-            fn(k & 1)
-        torch.cuda.synchronize()
-        # `iters` calls back to back between two events: the tensors (0.5 GB each at 2^28) are far larger than L2,
-        # and launch gaps overlap with the previous call's tail as they do inside a real step
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for k in range(iters):
-            fn(k & 1)
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / iters
-        out[name] = {"ms": round(ms, 4), "gbs": round(nbytes / ms / 1e6, 1)}
-    del xs, codes, backs
-    torch.cuda.empty_cache()
-    return out
+def per_label_ms(events):
+    """average device time per call label over the recorded steps"""
+    acc = {}
+    for row in events:
+        for (label, e0), (_, e1) in zip(row[:-1], row[1:]):
+            acc.setdefault(label, []).append(e0.elapsed_time(e1))
+    return {k: sum(v) / len(v) for k, v in acc.items()}
+
+
+def step_figures(step, avg):
+    """per-kernel figures of a step from its per-label average times: GEMM TFLOP/s, cast GB/s"""
+    gemms = {k: round(step.flops_per_gemm / (avg[k] * 1e-3) / 1e12, 1) for k in avg if k.startswith("gemm_")}
+    casts = {}
+    for k in avg:
+        if k.startswith("quantize_current"):
+            casts[k] = round(5.0 * step.cast_elements(k) / (avg[k] * 1e-3) / 1e9, 1)
+        elif k == "dequantize":
+            casts[k] = round(3.0 * step.cast_elements(k) / (avg[k] * 1e-3) / 1e9, 1)
+    gemm_ms = sum(avg[k] for k in gemms) / max(1, len(gemms))
+    cast_ms = sum(avg[k] for k in casts)
+    total = sum(avg.values())
+    return {"gemm_tflops": gemms, "cast_gbs": casts,
+            "gemm_mean_tflops": step.flops_per_gemm / (gemm_ms * 1e-3) / 1e12,
+            "cast_total_gbs": step.cast_bytes / (cast_ms * 1e-3) / 1e9,
+            "kernels": {k: {"avg_ms": round(v, 4), "share": round(v / total, 4)} for k, v in avg.items()}}
 
 
 def bench_cast_sizes(torch, api, synth, device, pk, sizes=(20, 24, 28, 30)):
@@ -240,7 +247,8 @@ def bench_cast_sizes(torch, api, synth, device, pk, sizes=(20, 24, 28, 30)):
      - "same_buffer": 20 back-to-back calls on one tensor; below ~126 MB of traffic the tensor stays in L2, so the
        figure is flagged l2_resident and is a latency / L2 number, not an HBM one;
      - "ring": a CUDA graph of calls that walk a ring of distinct tensors totalling more than 512 MB, so that every
-       call misses L2: the HBM-honest figure for the small sizes (and the launch cost without host gaps)."""
+       call misses L2: the HBM-honest figure for the small sizes (and the launch cost without host gaps).
+    Calls of a few microseconds are bound by launch latency, not by HBM: flagged latency_bound."""
     out = {}
     sc = torch.tensor([3.0, 1.0 / 3.0, 0.0, 0.0, 0.0], dtype=torch.float32, device=device)
     s, si, a, s2, si2 = sc[0:1], sc[1:2], sc[2:3], sc[3:4], sc[4:5]
@@ -259,8 +267,10 @@ def bench_cast_sizes(torch, api, synth, device, pk, sizes=(20, 24, 28, 30)):
         cases = {
             "amax": (lambda i: api.fp8_amax(xs[i], a), 2.0 * n),
             "quantize_e4m3_with_amax": (lambda i: api.fp8_quantize(xs[i], api.E4M3, s, cs[i], api.SATURATE, a), 3.0 * n),
+            "quantize_e5m2_with_amax": (lambda i: api.fp8_quantize(xs[i], api.E5M2, s, cs[i], api.SATURATE, a), 3.0 * n),
             "quantize_current_e4m3": (lambda i: api.fp8_quantize_current(xs[i], api.E4M3, cs[i], a, s2, si2), 5.0 * n),
             "dequantize_e4m3": (lambda i: api.fp8_dequantize(cs[i], api.E4M3, si, bs[i]), 3.0 * n),
+            "fake_quantize_e4m3": (lambda i: api.fp8_fake_quantize(xs[i], api.E4M3, s, si, bs[i]), 4.0 * n),
         }
         row = {"ring_tensors": ring}
         for name, (fn, nbytes) in cases.items():
@@ -296,7 +306,8 @@ def bench_cast_sizes(torch, api, synth, device, pk, sizes=(20, 24, 28, 30)):
             torch.cuda.synchronize()
             gms = e0.elapsed_time(e1) / calls
             entry["ring"] = {"us": round(gms * 1e3, 2), "gbs": round(nbytes / gms / 1e6, 1),
-                             "frac_of_measured_hbm": round(nbytes / gms / 1e6 / pk["hbm_gbs"], 4), "calls_in_graph": calls}
+                             "frac_of_measured_hbm": round(nbytes / gms / 1e6 / pk["hbm_gbs"], 4), "calls_in_graph": calls,
+                             "latency_bound": bool(gms * 1e3 < 8.0)}
             del graph
             row[name] = entry
         out["2pow%d" % log2n] = row
@@ -305,147 +316,73 @@ def bench_cast_sizes(torch, api, synth, device, pk, sizes=(20, 24, 28, 30)):
     return out
 
 
-def bench_config(torch, api, synth, device, pk, which):
-    """One of the five named workloads, every call timed alone (20 back-to-back launches after a short idle):
-    1 = 256 x 256 fp32 tensors, casts and a 256^3 GEMM (latency-bound); 2 = the cast size sweep; 3 = hidden-4096
-    forward (casts of X and W, forward GEMM); 4 = hidden-4096 backward (cast of dY, dgrad, wgrad); 5 = the
-    175B-class FFN, hidden 12288 (casts of X, W, dY; forward and dgrad GEMMs)."""
-    if which == 2:
-        return bench_cast_sizes(torch, api, synth, device, pk)
-
-    def timed(fn, n=20):
-        torch.cuda.synchronize()
-        time.sleep(0.25)
-        for _ in range(3):
-            fn()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(n):
-            fn()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / n
-
-    bf, f32, u8 = torch.bfloat16, torch.float32, torch.uint8
-    E4, E5, KM, MN = api.E4M3, api.E5M2, api.MAJOR_K, api.MAJOR_MN
-    out = {}
-
-    def cast(name, x, fmt):
-        q = torch.empty(x.shape, dtype=u8, device=device)
-        s = torch.zeros(3, dtype=f32, device=device)
-        esz = x.element_size()
-        ms = timed(lambda: api.fp8_quantize_current(x, fmt, q, s[0:1], s[1:2], s[2:3]))
-        nbytes = (2 * esz + 1.0) * x.numel()
-        out["quantize_current_" + name] = {"ms": round(ms, 4), "gbs": round(nbytes / ms / 1e6, 1),
-                                           "frac_of_measured_hbm": round(nbytes / ms / 1e6 / pk["hbm_gbs"], 4)}
-        return q, s[2:3]
-
-    def gemm(name, A, fa, ma, B, fb, mb, M, N, K, si_a, si_b, dtype=bf, n=20):
-        D = torch.empty(M, N, dtype=dtype, device=device)
-        am = torch.zeros(1, dtype=f32, device=device)
-        ms = timed(lambda: api.fp8_gemm(A, fa, ma, B, fb, mb, D, si_a, si_b, am), n)
-        tf = 2.0 * M * N * K / ms / 1e9
-        out["gemm_" + name] = {"ms": round(ms, 4), "tflops": round(tf, 1), "frac_of_2x_measured_bf16_burst": round(tf / (2 * pk["bf16_burst"]), 4),
-                               "frac_of_nominal_4500": round(tf / 4500.0, 4)}
-
-    if which == 1:
-        A = synth.normal_with_scaled_outliers(256 * 256, 0, synth.A_ID, 0.005, 64.0, dtype=f32, device=device).view(256, 256)
-        B = synth.normal_with_scaled_outliers(256 * 256, 0, synth.B_ID, 0.005, 64.0, dtype=f32, device=device).view(256, 256)
-        Aq, sia = cast("A_256x256_fp32", A, E4)
-        Bq, sib = cast("B_256x256_fp32", B, E4)
-        gemm("256x256x256_fp32_out", Aq, E4, KM, Bq, E4, KM, 256, 256, 256, sia, sib, dtype=f32)
-    elif which in (3, 4):
-        T, I, O = TOKENS, D_IN, D_OUT
-        X = synth.activations(T * I, 3, device=device).view(T, I)
-        W = synth.weights(I * O, 3, W_SIGMA, device=device).view(I, O)
-        Xq, six = cast("X_8192x4096", X, E4)
-        Wq, siw = cast("W_4096x16384", W, E4)
-        del X, W
-        if which == 3:
-            gemm("fprop_8192x16384x4096", Xq, E4, KM, Wq, E4, MN, T, O, I, six, siw)
-        else:
-            dY = synth.gradients(T * O, 4, device=device).view(T, O)
-            Gq, sig = cast("dY_8192x16384", dY, E5)
-            del dY
-            gemm("dgrad_8192x4096x16384", Gq, E5, KM, Wq, E4, KM, T, I, O, sig, siw)
-            gemm("wgrad_4096x16384x8192", Xq, E4, MN, Gq, E5, MN, I, O, T, six, sig)
-    elif which == 5:
-        T, I, O = 8192, 12288, 49152
-        X = synth.activations(T * I, 5, device=device).view(T, I)
-        Xq, six = cast("X_8192x12288", X, E4)
-        del X
-        W = synth.weights(I * O, 5, 0.006, device=device).view(I, O)
-        Wq, siw = cast("W_12288x49152", W, E4)
-        del W
-        dY = synth.gradients(T * O, 5, device=device).view(T, O)
-        Gq, sig = cast("dY_8192x49152", dY, E5)
-        del dY
-        torch.cuda.empty_cache()
-        gemm("fprop_8192x49152x12288", Xq, E4, KM, Wq, E4, MN, T, O, I, six, siw, n=5)
-        gemm("dgrad_8192x12288x49152", Gq, E5, KM, Wq, E4, KM, T, I, O, sig, siw, n=5)
-    else:
-        raise SystemExit("--config takes 1..5")
-    return out
-
-
-def bench_gemm_alone(torch, step, seconds=2.0):
-    """The forward GEMM of the step by itself: best single launch (burst) and a back-to-back loop of at
-    least `seconds` (sustained, under the power cap)."""
-    call = dict(step.calls())["gemm_fprop"]
-    flops = 2.0 * step.T * step.I * step.O
-    for _ in range(3):
-        call()
+def timed_alone(torch, fn, n=20):
+    """mean of n back-to-back calls after a short idle and three warm-up calls: a kernel timed by itself (burst)"""
     torch.cuda.synchronize()
-    best = 1e9
-    for _ in range(10):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(); call(); e1.record()
-        torch.cuda.synchronize()
-        best = min(best, e0.elapsed_time(e1))
-    n = max(10, int(seconds * 1e3 / best))
+    time.sleep(0.25)
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(n):
-        call()
+        fn()
     e1.record()
     torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / n
-    return {"shape": "M=%d N=%d K=%d, E4M3 x E4M3 -> bf16" % (step.T, step.O, step.I),
-            "burst_tflops": round(flops / best / 1e9, 1), "sustained_tflops": round(flops / ms / 1e9, 1),
-            "sustained_launches": n, "sustained_seconds": round(ms * n / 1e3, 2)}
+    return e0.elapsed_time(e1) / n
+
+
+def bench_layer_alone(torch, step, pk, n_gemm=20):
+    """Every call of a layer's step timed by itself (burst regime), with its roofline fraction:
+    GEMMs against 2 x the measured bf16 burst rate, casts against the measured copy bandwidth."""
+    out = {}
+    for label, fn in step.calls():
+        if label.startswith("gemm_"):
+            ms = timed_alone(torch, fn, n_gemm)
+            tf = step.flops_per_gemm / ms / 1e9
+            out[label] = {"ms": round(ms, 4), "tflops": round(tf, 1), "frac_of_2x_measured_bf16_burst": round(tf / (2 * pk["bf16_burst"]), 4),
+                          "frac_of_nominal_4500": round(tf / NOMINAL_FP8_TFLOPS, 4)}
+        else:
+            ms = timed_alone(torch, fn)
+            nbytes = (5.0 if label.startswith("quantize_current") else 3.0) * step.cast_elements(label)
+            out[label] = {"ms": round(ms, 4), "gbs": round(nbytes / ms / 1e6, 1), "frac_of_measured_hbm": round(nbytes / ms / 1e6 / pk["hbm_gbs"], 4),
+                          "frac_of_nominal_8000": round(nbytes / ms / 1e6 / NOMINAL_HBM_GBS, 4)}
+    return out
+
+
+def bench_tiny(torch, api, synth, device):
+    """The 256 x 256 fp32 tensors of the smallest workload: casts and a 256^3 GEMM, every call latency-bound."""
+    f32, u8 = torch.float32, torch.uint8
+    out = {}
+    A = synth.normal_with_scaled_outliers(256 * 256, 0, synth.A_ID, 0.005, 64.0, dtype=f32, device=device).view(256, 256)
+    B = synth.normal_with_scaled_outliers(256 * 256, 0, synth.B_ID, 0.005, 64.0, dtype=f32, device=device).view(256, 256)
+    q, sc = [], []
+    for name, x in (("A", A), ("B", B)):
+        c = torch.empty(256, 256, dtype=u8, device=device)
+        s = torch.zeros(3, dtype=f32, device=device)
+        ms = timed_alone(torch, lambda: api.fp8_quantize_current(x, api.E4M3, c, s[0:1], s[1:2], s[2:3]))
+        out["quantize_current_%s_256x256_fp32" % name] = {"us": round(ms * 1e3, 2), "latency_bound": True}
+        q.append(c); sc.append(s)
+    D = torch.empty(256, 256, dtype=f32, device=device)
+    am = torch.zeros(1, dtype=f32, device=device)
+    ms = timed_alone(torch, lambda: api.fp8_gemm(q[0], api.E4M3, api.MAJOR_K, q[1], api.E4M3, api.MAJOR_K, D, sc[0][2:3], sc[1][2:3], am))
+    out["gemm_256x256x256_fp32_out"] = {"us": round(ms * 1e3, 2), "latency_bound": True,
+                                        "note": "host time of one call included: the launches are issued back to back from Python"}
+    return out
 
 
 def bench_next_rows(torch, api, synth, device, pk, iters=5):
     """The rows beyond the core path, each timed alone on workload-shaped tensors: simulated-FP8 round trip,
     per-channel weight scales, FP8-output GEMM, attention-style batched GEMM."""
     def timed(fn):
-        """mean of `iters` groups of 4 back-to-back calls (launch gaps overlap the previous call, as inside a step);
-        a short idle first, so that each kernel is timed alone and not in the power state its predecessor left"""
-        torch.cuda.synchronize()
-        time.sleep(0.25)
-        for _ in range(3):
-            fn()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(4 * iters):
-            fn()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / (4 * iters)
+        return timed_alone(torch, fn, 4 * iters)
 
+    L = LAYERS["hidden4096"]
+    TOKENS, D_IN, D_OUT, W_SIGMA = L["tokens"], L["d_in"], L["d_out"], L["w_sigma"]
     out = {}
     f32 = torch.float32
     sc = torch.tensor([3.0, 1.0 / 3.0, 0.0, 0.0], dtype=f32, device=device)
     s, si, a = sc[0:1], sc[1:2], sc[2:3]
-    # simulated FP8 (quantize + dequantize in one pass), 2^28 bf16 elements: 4 B per element
-    n = 1 << 28
-    x = synth.normal_laplace_mixture(n, 1, synth.T_ID, device=device)
-    y = torch.empty_like(x)
-    ms = timed(lambda: api.fp8_fake_quantize(x, api.E4M3, s, si, y))
-    out["fake_quantize_e4m3_2pow28"] = {"ms": round(ms, 4), "gbs": round(4.0 * n / ms / 1e6, 1), "frac_of_measured_hbm": round(4.0 * n / ms / 1e6 / pk["hbm_gbs"], 4)}
-    del x, y
     # per-channel weight scales on W [4096 x 16384] bf16, one channel per output column
     W = synth.weights(D_IN * D_OUT, 3, W_SIGMA, device=device).view(D_IN, D_OUT)
     am = torch.empty(D_OUT, dtype=f32, device=device)
@@ -477,29 +414,16 @@ def bench_next_rows(torch, api, synth, device, pk, iters=5):
     out["gemm_fprop_channel_scales"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
     ms = timed(lambda: api.fp8_gemm_fp8out(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Yq, api.E4M3, sx[2:3], si, s, a))
     out["gemm_fprop_fp8_output"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
-    # split accumulation (partial sums every 2048 of K added in registers): forward K = 4096 and, on the same codes
-    # read as dY-shaped operands, the dgrad shape K = 16384
-    ms = timed(lambda: api.fp8_gemm(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, sx[2:3], si, a, acc=api.ACC_SPLIT))
-    out["gemm_fprop_split_accumulation"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
+    # split accumulation (partial sums every 2048 of K added in registers) against one accumulator, same codes:
+    # forward K = 4096 and, on the same codes read as dY-shaped operands, the dgrad shape K = 16384
+    for name, acc in (("one_accumulator", api.ACC_FAST), ("split_accumulation", api.ACC_SPLIT)):
+        ms = timed(lambda: api.fp8_gemm(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, sx[2:3], si, a, acc=acc))
+        out["gemm_fprop_K4096_" + name] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
     dX = torch.empty(TOKENS, D_IN, dtype=torch.bfloat16, device=device)
-    ms = timed(lambda: api.fp8_gemm(Yq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, si, si, a, acc=api.ACC_SPLIT))
-    out["gemm_dgrad_split_accumulation"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
-    ms = timed(lambda: api.fp8_gemm(Yq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, si, si, a))
-    out["gemm_dgrad_same_codes_one_accumulator"] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
-    del dX
-    del W, X, Y, Yq
-    # a weight-bandwidth-bound product with few output tiles: 16 rows against W^T stored [4096 x 16384] (K = 16384),
-    # plain and with the contraction cut into slices
-    Xs = torch.randint(0, 0x78, (16, D_OUT), dtype=torch.uint8, device=device)
-    Wt = torch.randint(0, 0x78, (D_IN, D_OUT), dtype=torch.uint8, device=device)          # [N = 4096, K = 16384], K-major
-    Ys = torch.empty(16, D_IN, dtype=torch.bfloat16, device=device)
-    sp, nb = api.fp8_gemm_splitk_workspace(16, D_IN, D_OUT)
-    ws = torch.empty(max(nb // 4, 4), dtype=f32, device=device)
-    ms = timed(lambda: api.fp8_gemm(Xs, api.E4M3, api.MAJOR_K, Wt, api.E4M3, api.MAJOR_K, Ys, si, si, a))
-    out["gemm_16x4096x16384_one_launch"] = {"ms": round(ms, 4), "weight_gbs": round(D_IN * D_OUT / ms / 1e6, 1)}
-    ms = timed(lambda: api.fp8_gemm_splitk(Xs, api.E4M3, api.MAJOR_K, Wt, api.E4M3, api.MAJOR_K, Ys, si, si, ws if nb else None, a))
-    out["gemm_16x4096x16384_splitk"] = {"ms": round(ms, 4), "weight_gbs": round(D_IN * D_OUT / ms / 1e6, 1), "splits": sp}
-    del Xs, Wt, Ys, ws
+    for name, acc in (("one_accumulator", api.ACC_FAST), ("split_accumulation", api.ACC_SPLIT)):
+        ms = timed(lambda: api.fp8_gemm(Yq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, si, si, a, acc=acc))
+        out["gemm_dgrad_K16384_" + name] = {"ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1)}
+    del dX, W, X, Y, Yq
     # attention-style batched products: 32 heads, 4096 tokens, head dim 128: scores = Q.K^T, context = P.V
     H, S, Dh = 32, 4096, 128
     Q = torch.randint(0, 0x78, (H, S, Dh), dtype=torch.uint8, device=device)
@@ -525,7 +449,7 @@ def bench_next_rows(torch, api, synth, device, pk, iters=5):
 _oracle_inputs = {}
 
 
-def oracle_step(sample_tokens: int, threads: int, sample_out: int = D_OUT):
+def oracle_step(layer: str, sample_tokens: int, threads: int, sample_out: int | None = None):
     """The same step on a bounded sample of the layer: `sample_tokens` tokens and `sample_out` output features
     (W is [d_in, sample_out], same recipe), run by the CPU oracle as it stands.
     Returns (seconds, gemm flops of the sample)."""
@@ -535,17 +459,18 @@ def oracle_step(sample_tokens: int, threads: int, sample_out: int = D_OUT):
     import oracle
     from paper_2209_05433_b200 import synth
 
-    T, I, O = sample_tokens, D_IN, sample_out
+    L = LAYERS[layer]
+    T, I, O = sample_tokens, L["d_in"], sample_out or L["d_out"]
 
     def bits(t):
         return t.view(torch.int16).numpy().view(np.uint16)
 
-    key = (T, O)
+    key = (layer, T, O)
     if key not in _oracle_inputs:                                  # synthetic inputs are made once, outside the timed part
         _oracle_inputs.clear()
-        _oracle_inputs[key] = (bits(synth.activations(T * I, 3, dtype=torch.bfloat16)),
-                               bits(synth.weights(I * O, 3, W_SIGMA, dtype=torch.bfloat16)),
-                               bits(synth.gradients(T * O, 4, dtype=torch.bfloat16)))
+        _oracle_inputs[key] = (bits(synth.activations(T * I, L["seed"], dtype=torch.bfloat16)),
+                               bits(synth.weights(I * O, L["seed"], L["w_sigma"], dtype=torch.bfloat16)),
+                               bits(synth.gradients(T * O, L["seed"], dtype=torch.bfloat16)))
     X, W, dY = _oracle_inputs[key]
     t0 = time.perf_counter()
     q, sinv = {}, {}
@@ -553,48 +478,53 @@ def oracle_step(sample_tokens: int, threads: int, sample_out: int = D_OUT):
         s, si = oracle.scale_from_amax(oracle.amax(t, threads), fmt)
         q[name], sinv[name] = oracle.quantize(t, s, fmt, threads=threads), si
     oracle.dequantize(q["x"], sinv["x"], oracle.E4M3, "bf16", threads=threads)
-    y, _ = oracle.gemm_rows(q["x"], oracle.E4M3, (I, 1), q["w"], oracle.E4M3, (O, 1), O, I, 0, T, sinv["x"], sinv["w"], threads)
-    dx, _ = oracle.gemm_rows(q["g"], oracle.E5M2, (O, 1), q["w"], oracle.E4M3, (1, O), I, O, 0, T, sinv["g"], sinv["w"], threads)
-    dw, _ = oracle.gemm_rows(q["x"], oracle.E4M3, (1, I), q["g"], oracle.E5M2, (O, 1), O, T, 0, I, sinv["x"], sinv["g"], threads)
-    for r in (y, dx, dw):
+    results = []
+    if "fprop" in L["passes"]:
+        results.append(oracle.gemm_rows(q["x"], oracle.E4M3, (I, 1), q["w"], oracle.E4M3, (O, 1), O, I, 0, T, sinv["x"], sinv["w"], threads)[0])
+    if "dgrad" in L["passes"]:
+        results.append(oracle.gemm_rows(q["g"], oracle.E5M2, (O, 1), q["w"], oracle.E4M3, (1, O), I, O, 0, T, sinv["g"], sinv["w"], threads)[0])
+    if "wgrad" in L["passes"]:
+        results.append(oracle.gemm_rows(q["x"], oracle.E4M3, (1, I), q["g"], oracle.E5M2, (O, 1), O, T, 0, I, sinv["x"], sinv["g"], threads)[0])
+    for r in results:
         oracle.round_bf16_from_f64(r)
     dt = time.perf_counter() - t0
-    return dt, 3 * 2.0 * T * I * O
+    return dt, len(results) * 2.0 * T * I * O
 
 
-def reference_sample(steps: int, warmup: int, threads: int):
-    """(tokens, output features) of the per-step sample: 8 tokens and as many output features (multiples of
-    256) as fit about 150 s for the whole run, at most the full layer (about 6 s per step on 8 cores).
-    Every cost of the step (weight cast, three GEMMs, wgrad outputs) is linear in the feature count."""
-    t_small, _ = oracle_step(8, threads, 256)                      # calibration on the smallest sample
+def reference_sample(layer: str, steps: int, warmup: int, threads: int):
+    """(tokens, output features) of the per-step sample: 4 tokens and as many output features (multiples of
+    256) as fit about 150 s for the whole run, at most the full layer.
+    Every cost of the step (weight cast, the GEMMs) is linear in the feature count."""
+    t_small, _ = oracle_step(layer, 4, threads, 256)               # calibration on the smallest sample
     total = float(os.environ.get("FP8_BENCH_REFERENCE_SECONDS", "150"))      # wall-clock aim for the whole run
     budget = min(8.0, total / max(1, steps + warmup))
     grow = max(1.0, budget / max(t_small, 1e-3))
-    sample_out = int(min(D_OUT, 256 * int(grow)))
-    return 8, max(256, sample_out // 256 * 256)
+    sample_out = int(min(LAYERS[layer]["d_out"], 256 * int(grow)))
+    return 4, max(256, sample_out // 256 * 256)
 
 
-def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
+def run_reference(args, world, rank):
     if rank != 0:
-        return
+        return                                                     # the oracle runs once, on rank 0's host cores
+    layer = HEADLINE
+    L = LAYERS[layer]
     threads = os.cpu_count() or 1
-    sample_tokens, sample_out = reference_sample(args.steps, args.warmup, threads)
+    sample_tokens, sample_out = reference_sample(layer, args.steps, args.warmup, threads)
     for _ in range(args.warmup):
-        oracle_step(sample_tokens, threads, sample_out)
+        oracle_step(layer, sample_tokens, threads, sample_out)
     times, flops = [], 0.0
     for _ in range(args.steps):
-        dt, flops = oracle_step(sample_tokens, threads, sample_out)
+        dt, flops = oracle_step(layer, sample_tokens, threads, sample_out)
         times.append(dt)
     total = sum(times)
     value = flops * len(times) / total / 1e12
     sample = "the same step on %d of the %d tokens and %d of the %d output features, CPU oracle as it stands" % (
-        sample_tokens, TOKENS, sample_out, D_OUT)
+        sample_tokens, L["tokens"], sample_out, L["d_out"])
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64 accumulation over decoded fp8 codes", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample": sample},
+        "config": {"workload": workload_text(layer), "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -606,62 +536,84 @@ def run_reference(args):
 # our arm
 # ----------------------------------------------------------------------------
 
-def run_ours(args):
+def run_only(args, torch, api, synth, device):
+    """One call of a layer's step, alone (what the ncu captures under profiles/ run): a full step first to set
+    scales and codes, then `--steps` launches of the named call."""
+    step = LinearStep(torch, api, synth, device, args.layer)
+    step.run()
+    for _ in range(max(args.warmup, 1)):
+        step.run(args.only)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step.run(args.only)
+    e1.record()
+    torch.cuda.synchronize()
+    st, detail = api.fp8_async_status()
+    if st != 0:
+        raise SystemExit("device-side wait expired (code %d)" % detail)
+    print(json.dumps({"only": args.only, "layer": args.layer, "steps": args.steps, "ms_per_call": e0.elapsed_time(e1) / args.steps}))
+
+
+def run_ours(args, world, rank, local):
     import torch
     import torch.distributed as dist
 
     from paper_2209_05433_b200 import api, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    if local >= torch.cuda.device_count():
+        raise SystemExit("rank %d has no GPU: %d visible" % (local, torch.cuda.device_count()))
     torch.cuda.set_device(local)
     device = "cuda:%d" % local
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device(device))
     api.load()
+    pk = peaks()
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    if args.cast_sizes_only:
-        print(json.dumps({"cast_sizes": bench_cast_sizes(torch, api, synth, device, peaks())}))
+    def max_over_ranks(ms):
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return ms
+
+    if args.only:
+        run_only(args, torch, api, synth, device)
         return
     if args.config:
-        print(json.dumps({"config": args.config, "results": bench_config(torch, api, synth, device, peaks(), args.config)}))
+        if args.config == 1:
+            res = bench_tiny(torch, api, synth, device)
+        elif args.config == 2:
+            res = bench_cast_sizes(torch, api, synth, device, pk)
+        elif args.config in (3, 4, 5):
+            res = bench_layer_alone(torch, LinearStep(torch, api, synth, device, "hidden12288" if args.config == 5 else "hidden4096"), pk,
+                                    n_gemm=5 if args.config == 5 else 20)
+        else:
+            raise SystemExit("--config takes 1..5")
+        print(json.dumps({"config": args.config, "results": res}))
         return
-    if args.next_rows_only:
-        # profiling aid: only the kernels beyond the core path, each on workload-shaped tensors
-        print(json.dumps({"next_rows": bench_next_rows(torch, api, synth, device, peaks(), iters=max(1, min(args.steps, 5)))}))
-        return
+
     # independent batches per rank: no data-path collective (per-tensor amax is local to a rank's own tensors)
-    step = LinearStep(torch, api, synth, device, seed=3 + 16 * rank, fused_cast=not args.unfused_cast)
-    if args.only:
-        # profiling aid: one full step to set the scales and codes, then only the named call, timed alone
-        step.run()
-        for _ in range(max(args.warmup, 1)):
-            step.run(args.only)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            step.run(args.only)
-        e1.record()
-        torch.cuda.synchronize()
-        print(json.dumps({"only": args.only, "steps": args.steps, "ms_per_step": e0.elapsed_time(e1) / args.steps}))
-        return
-    for _ in range(max(args.warmup, 3)):
+    layer = HEADLINE
+    step = LinearStep(torch, api, synth, device, layer, seed_offset=16 * rank)
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
         step.run()
     barrier()
     st, detail = api.fp8_async_status()
     if st != 0:
         raise SystemExit("device-side wait expired during warm-up (code %d)" % detail)
 
+    # ---- the K timed steps
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -673,26 +625,35 @@ def run_ours(args):
         step.run_timed(events)
     barrier()
     launches = api.fp8_launch_count() - launches0
-    total_ms = events[0][0][1].elapsed_time(events[-1][-1][1])
-    per_label = {}
-    for row in events:
-        for (label, e0), (_, e1) in zip(row[:-1], row[1:]):
-            per_label.setdefault(label, []).append(e0.elapsed_time(e1))
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(events[0][0][1].elapsed_time(events[-1][-1][1]))
+    avg = per_label_ms(events)
     clocks = sampler.stop() if rank == 0 else None
     st, detail = api.fp8_async_status()
     if st != 0:
         raise SystemExit("device-side wait expired during the timed region (code %d)" % detail)
 
+    # ---- sustained: whole steps back to back for at least two seconds, clocks sampled over exactly that loop
+    ms_per_step = total_ms / args.steps
+    n_sus = max(args.steps, int(args.sustained_seconds * 1e3 / ms_per_step) + 1)
+    sampler2 = ClockSampler(local)
+    if rank == 0:
+        sampler2.start()
+    sus_events = []
+    barrier()
+    for _ in range(n_sus):
+        step.run_timed(sus_events)
+    barrier()
+    sus_ms = max_over_ranks(sus_events[0][0][1].elapsed_time(sus_events[-1][-1][1]))
+    sus_avg = per_label_ms(sus_events[len(sus_events) // 4:])      # per-kernel figures from the last three quarters: clocks have settled
+    sus_clocks = sampler2.stop() if rank == 0 else None
+    del events, sus_events
+
     # ---- end to end: pinned host inputs -> device, the step, results -> pinned host, EVERY step.
     # Three streams (copy in, compute, copy out) and two device buffer sets, so that the upload of step i+1 and
     # the download of step i-1 overlap the kernels of step i; each step still moves all of its own bytes.
-    steps2 = [step, LinearStep(torch, api, synth, device, seed=3 + 16 * rank, fused_cast=not args.unfused_cast)]
-    host_in = [torch.empty(t.shape, dtype=t.dtype).pin_memory().copy_(t) for t in (step.X, step.W, step.dY)]
-    host_out = [[torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (st.Y, st.dX, st.dW)] for st in steps2]
+    steps2 = [step, LinearStep(torch, api, synth, device, layer, seed_offset=16 * rank)]
+    host_in = [torch.empty(t.shape, dtype=t.dtype).pin_memory().copy_(t) for t in step.inputs]
+    host_out = [[torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in s_.outputs] for s_ in steps2]
     host_scal = [torch.empty(16, dtype=torch.float32).pin_memory() for _ in steps2]
     h2d = sum(t.numel() * t.element_size() for t in host_in)
     d2h = sum(t.numel() * t.element_size() for t in host_out[0]) + host_scal[0].numel() * 4
@@ -707,25 +668,25 @@ def run_ours(args):
 
     def e2e_step(i):
         b = i & 1
-        st = steps2[b]
+        sb = steps2[b]
         with torch.cuda.stream(s_in):
             s_in.wait_event(ev_comp[b])                  # the previous step on this set has consumed its inputs
-            for h, d in zip(host_in, (st.X, st.W, st.dY)):
+            for h, d in zip(host_in, sb.inputs):
                 d.copy_(h, non_blocking=True)
             ev_in[b].record(s_in)
         with torch.cuda.stream(s_comp):
             s_comp.wait_event(ev_in[b])
             s_comp.wait_event(ev_out[b])                 # its previous outputs have left the device buffers
-            st.run()
+            sb.run()
             ev_comp[b].record(s_comp)
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_comp[b])
-            for h, d in zip(host_out[b], (st.Y, st.dX, st.dW)):
+            for h, d in zip(host_out[b], sb.outputs):
                 h.copy_(d, non_blocking=True)
-            host_scal[b].copy_(st.scal, non_blocking=True)
+            host_scal[b].copy_(sb.scal, non_blocking=True)
             ev_out[b].record(s_out)
 
-    e2e_steps = max(2, min(args.steps, 10))
+    e2e_steps = max(2, min(args.steps, 6))
     for i in range(2):
         e2e_step(i)
     barrier()
@@ -737,81 +698,94 @@ def run_ours(args):
     s_out.wait_stream(s_in)
     e1.record(s_out)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1))
+    del steps2[1], host_in, host_out
+    torch.cuda.empty_cache()
 
     if rank == 0:
-        pk = peaks()
-        ms_per_step = total_ms / args.steps
         value = step.gemm_flops * world / (ms_per_step * 1e-3) / 1e12
-        avg = {k: sum(v) / len(v) for k, v in per_label.items()}
-        calls_per_step = {k: len(v) // args.steps for k, v in per_label.items()}
-        step_sum = sum(avg[k] * calls_per_step[k] for k in avg)
-        kernels = {k: {"avg_ms": round(avg[k], 4), "calls_per_step": calls_per_step[k],
-                       "share": round(avg[k] * calls_per_step[k] / step_sum, 4)} for k in avg}
-        # dominant kernel: the FP8 GEMM (three launches per step of 2*T*I*O flops each)
-        gemm_ms = (avg["gemm_fprop"] + avg["gemm_dgrad"] + avg["gemm_wgrad"]) / 3.0
-        gemm_flops = 2.0 * TOKENS * D_IN * D_OUT
-        achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12
-        fp8_peak = 2.0 * pk["bf16_sustained"]            # fp8 : bf16 nominal ratio is 2
-        roofline = {"bound": "tensor", "kernel": "k_gemm_fp8", "achieved": round(achieved, 1), "peak": round(fp8_peak, 1),
-                    "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4), "traffic": NCU_TRAFFIC_GEMM_BYTES,
-                    "traffic_note": "DRAM bytes per launch, ncu capture of the forward GEMM (profiles/gemm_fp8_forward_hidden4096.md); algorithmic 3.69e8",
-                    "peak_source": "2 x %s bf16 sustained cuBLAS TFLOP/s (fp8:bf16 nominal ratio)" % pk["source"],
-                    "frac_of_nominal_4500": round(achieved / NOMINAL_FP8_TFLOPS, 4),
-                    "per_gemm_tflops": {k: round(gemm_flops / (avg[k] * 1e-3) / 1e12, 1) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}}
+        burst = step_figures(step, avg)
+        sus = step_figures(step, sus_avg)
+        sus_ms_per_step = sus_ms / n_sus
+        sms = torch.cuda.get_device_properties(local).multi_processor_count
+        traffic = ncu_traffic()
+
+        def clock_normalised(tflops, mhz):
+            """fraction of the tensor pipes' rate at the clock the loop ran at: flop / (SMs x 8192 MAC x 2 x clock)"""
+            if not mhz:
+                return None
+            return round(tflops * 1e12 / (sms * FP8_MACS_PER_SM_PER_CLOCK * 2.0 * mhz * 1e6), 4)
+
+        # dominant kernel: the FP8 GEMM (launches of 2*T*I*O flops each).  frac: sustained figure / sustained peak.
+        fp8_sus, fp8_burst = 2.0 * pk["bf16_sustained"], 2.0 * pk["bf16_burst"]         # fp8 : bf16 nominal ratio is 2
+        a_sus, a_burst = sus["gemm_mean_tflops"], burst["gemm_mean_tflops"]
+        roofline = {
+            "bound": "tensor", "kernel": "k_gemm_fp8", "achieved": round(a_sus, 1), "peak": round(fp8_sus, 1), "unit": "TFLOP/s",
+            "frac": round(a_sus / fp8_sus, 4), "traffic": traffic.get("k_gemm_fp8.fprop." + layer),
+            "regime": "sustained: per-launch CUDA events inside a loop of %d whole steps (%.2f s), divided by 2 x %s bf16 sustained cuBLAS "
+                      "TFLOP/s (fp8:bf16 nominal ratio 2)" % (n_sus, sus_ms / 1e3, pk["source"]),
+            "algorithmic_flops_per_launch": step.flops_per_gemm,
+            "per_gemm_tflops": sus["gemm_tflops"],
+            "clock_normalised": {"sm_mhz_median": sus_clocks["sm_mhz"], "frac_of_tensor_pipe_rate": clock_normalised(a_sus, sus_clocks["sm_mhz"]),
+                                 "formula": "flop / (%d SMs x %d MAC x 2 x median SM clock of the loop)" % (sms, FP8_MACS_PER_SM_PER_CLOCK)},
+            "burst": {"achieved": round(a_burst, 1), "peak": round(fp8_burst, 1), "frac": round(a_burst / fp8_burst, 4),
+                      "regime": "the %d timed steps (%.3f s), divided by 2 x %s bf16 burst cuBLAS TFLOP/s" % (args.steps, total_ms / 1e3, pk["source"]),
+                      "per_gemm_tflops": burst["gemm_tflops"]},
+            "frac_of_nominal_4500": round(a_sus / NOMINAL_FP8_TFLOPS, 4), "burst_frac_of_nominal_4500": round(a_burst / NOMINAL_FP8_TFLOPS, 4),
+            "traffic_note": "DRAM bytes per launch of the forward GEMM from the ncu capture summarised under profiles/; algorithmic %.3e"
+                            % (step.T * step.I + step.I * step.O + 2.0 * step.T * step.O),
+        }
         # the memory-bound half: amax + quantize (+ dequantize) of the step against HBM
-        cast_labels = [k for k in ("quantize_current", "amax", "scale", "quantize", "dequantize") if k in avg]
-        cast_ms = sum(avg[k] * calls_per_step[k] for k in cast_labels)
-        cast_gbs = step.cast_bytes / (cast_ms * 1e-3) / 1e9
-        n_x = TOKENS * D_IN + D_IN * D_OUT + TOKENS * D_OUT
-        roofline_cast = {"bound": "hbm", "kernel": "casts of the step: " + " + ".join(cast_labels), "achieved": round(cast_gbs, 1),
-                         "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": round(cast_gbs / pk["hbm_gbs"], 4),
-                         "traffic": NCU_TRAFFIC_QUANTIZE_CURRENT_BYTES if "quantize_current" in avg else None,
-                         "peak_source": pk["source"] + " copy bandwidth", "frac_of_nominal_8000": round(cast_gbs / NOMINAL_HBM_GBS, 4),
-                         "algorithmic_bytes": "5 B per bf16 element for amax+quantize (two reads, one write), 3 B per element for dequantize; "
-                                              "re-reads served by L2 still count as algorithmic bytes"}
-        if "quantize_current" in avg:
-            roofline_cast["quantize_current_gbs"] = round(5.0 * n_x / 3 / (avg["quantize_current"] * 1e-3) / 1e9, 1)
-        else:
-            roofline_cast["amax_gbs"] = round(2.0 * n_x / 3 / (avg["amax"] * 1e-3) / 1e9, 1)
-            roofline_cast["quantize_gbs"] = round(3.0 * n_x / 3 / (avg["quantize"] * 1e-3) / 1e9, 1)
-        cast = None
-        if not args.no_cast_sweep:
-            cast = bench_cast_sweep(torch, api, synth, device, args.cast_log2n)
-            for v in cast.values():
-                v["frac_of_measured_hbm"] = round(v["gbs"] / pk["hbm_gbs"], 4)
-        cast_sizes = bench_cast_sizes(torch, api, synth, device, pk) if world == 1 and not args.no_cast_sweep else None
-        gemm_alone = bench_gemm_alone(torch, step) if world == 1 and not args.no_next_rows else None
-        next_rows = None
-        if world == 1 and not args.no_next_rows:
+        c_sus, c_burst = sus["cast_total_gbs"], burst["cast_total_gbs"]
+        roofline_cast = {
+            "bound": "hbm", "kernel": "casts of the step: k_quantize_current (X, W, dY) + k_dequantize", "achieved": round(c_sus, 1),
+            "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": round(c_sus / pk["hbm_gbs"], 4),
+            "traffic": traffic.get("k_quantize_current.W." + layer),
+            "peak_source": pk["source"] + " copy bandwidth", "regime": "sustained loop (same as roofline)",
+            "per_call_gbs": sus["cast_gbs"], "burst": {"achieved": round(c_burst, 1), "frac": round(c_burst / pk["hbm_gbs"], 4), "per_call_gbs": burst["cast_gbs"]},
+            "frac_of_nominal_8000": round(c_sus / NOMINAL_HBM_GBS, 4),
+            "algorithmic_bytes": "5 B per bf16 element for amax+quantize (two reads, one write), 3 B per element for dequantize; "
+                                 "re-reads served by L2 still count as algorithmic bytes",
+        }
+        sustained = {"steps": n_sus, "seconds": round(sus_ms / 1e3, 3), "ms_per_step": round(sus_ms_per_step, 4),
+                     "value": round(step.gemm_flops * world / (sus_ms_per_step * 1e-3) / 1e12, 1), "unit": UNIT, "clocks": sus_clocks,
+                     "kernels": sus["kernels"]}
+        per_config = cast_sizes = next_rows = cpu = None
+        if world == 1 and not args.quick:
+            del step
+            torch.cuda.empty_cache()
+            cast_sizes = bench_cast_sizes(torch, api, synth, device, pk)
+            small = LinearStep(torch, api, synth, device, "hidden4096")
+            per_config = {
+                "1_tiny_256": bench_tiny(torch, api, synth, device),
+                "2_cast_sweep": "see cast_sizes",
+                "3_4_hidden4096_each_call_alone": bench_layer_alone(torch, small, pk),
+                "5_hidden12288": {"burst_in_step": {"gemm_tflops": burst["gemm_tflops"], "cast_gbs": burst["cast_gbs"]},
+                                  "sustained_in_step": {"gemm_tflops": sus["gemm_tflops"], "cast_gbs": sus["cast_gbs"]}},
+            }
+            del small
+            torch.cuda.empty_cache()
             next_rows = bench_next_rows(torch, api, synth, device, pk)
-        cpu = None
-        if world == 1 and not args.no_cpu_baseline:
             threads = os.cpu_count() or 1
-            cpu_tokens = 24                     # about 10-20 s of CPU work on 16 cores
-            dt, flops = oracle_step(cpu_tokens, threads)
+            cpu_tokens = 2 if threads >= 12 else 1                 # about 20 s of CPU work on 16 cores
+            dt, flops = oracle_step(layer, cpu_tokens, threads)
             cpu = {"value": flops / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": round(dt, 2),
-                   "sample": "the same step with %d of the %d tokens (weights at full size), CPU oracle as it stands" % (cpu_tokens, TOKENS)}
+                   "sample": "the same step with %d of the %d tokens (weights at full size), CPU oracle as it stands" % (cpu_tokens, LAYERS[layer]["tokens"])}
+        L = LAYERS[layer]
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "fp8 (e4m3/e5m2) operands, f32 accumulate, bf16 out", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "tokens": TOKENS, "d_in": D_IN, "d_out": D_OUT, "parallelism": "dp%d" % world,
-                       "l2": "inputs larger than L2 (step touches > 1 GB)", "weights_layout": "[d_in, d_out] row-major"},
+            "config": {"workload": workload_text(layer), "tokens": L["tokens"], "d_in": L["d_in"], "d_out": L["d_out"], "parallelism": "dp%d" % world,
+                       "l2": "inputs larger than L2 (step touches > 5 GB)", "weights_layout": "[d_in, d_out] row-major",
+                       "regime_of_value": "the K timed steps (burst clocks when K steps last well under a second); see `sustained`"},
             "clocks": clocks,
-            "e2e": {"value": step.gemm_flops * world / (e2e_ms / e2e_steps * 1e-3) / 1e12, "unit": UNIT,
+            "e2e": {"value": step_flops_e2e(L, world, e2e_ms / e2e_steps), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
                     "how": "pinned host buffers; upload, kernels and download of consecutive steps overlap on three streams"},
             "gpu_launches": int(launches), "gpu_launches_note": "kernels plus 4-byte memset nodes enqueued by the library in the timed region",
-            "roofline": roofline, "roofline_cast": roofline_cast, "kernels": kernels, "cast_sweep_2pow%d" % args.cast_log2n: cast,
-            "cast_sizes": cast_sizes,
-            "gemm_alone": gemm_alone,
-            "next_rows": next_rows,
-            "cpu_baseline": cpu,
+            "roofline": roofline, "roofline_cast": roofline_cast, "sustained": sustained, "kernels": burst["kernels"],
+            "per_config": per_config, "cast_sizes": cast_sizes, "next_rows": next_rows, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     if world > 1:
@@ -819,26 +793,41 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def step_flops_e2e(L, world, ms):
+    return len(L["passes"]) * 2.0 * L["tokens"] * L["d_in"] * L["d_out"] * world / (ms * 1e-3) / 1e12
+
+
+def spawn_ranks(n):
+    """--gpus N without a torchrun environment: start N ranks of this script, one per GPU"""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n), "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-cast-sweep", action="store_true")
-    ap.add_argument("--no-next-rows", action="store_true")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0, help="minimum length of the sustained whole-step loop")
+    ap.add_argument("--quick", action="store_true", help="the step only: no per-config, cast-size, next-row or CPU-baseline sections")
     ap.add_argument("--config", type=int, default=0, help="run one of the five named workloads (1..5), every call timed alone")
-    ap.add_argument("--cast-sizes-only", action="store_true", help="only the cast bandwidth sweep over 2^20 .. 2^30 elements")
-    ap.add_argument("--next-rows-only", action="store_true", help="profiling aid: run only the next-row kernels")
-    ap.add_argument("--cast-log2n", type=int, default=28)
-    ap.add_argument("--unfused-cast", action="store_true", help="amax, scale and quantize as three calls per tensor instead of fp8_quantize_current")
-    ap.add_argument("--only", default=None, help="profiling aid: time only the calls with this label (e.g. gemm_fprop, quantize, amax)")
+    ap.add_argument("--only", default=None, help="time only the calls with this label of a layer's step (e.g. gemm_fprop, quantize_current_W)")
+    ap.add_argument("--layer", choices=sorted(LAYERS), default=HEADLINE, help="layer of --only")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args.gpus)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
-        run_reference(args)
+        run_reference(args, world, rank)
     else:
-        run_ours(args)
+        run_ours(args, world, rank, local)
 
 
 if __name__ == "__main__":

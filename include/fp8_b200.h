@@ -104,8 +104,10 @@ fp8_status fp8_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_o
  *              caller.  It must hold zeros before the first call; every call leaves it zeroed again,
  *              so one buffer serves any number of calls on one stream.  Calls that may overlap on the
  *              GPU (different streams) need different workspaces.
- * The grid barrier is a bounded wait: if it expires nothing is written and fp8_async_status reports
- * FP8_ERR_TIMEOUT (the workspace must then be zeroed again by the caller).
+ * The grid barrier is a bounded wait (about two seconds).  If it expires in any block, fp8_async_status
+ * reports FP8_ERR_TIMEOUT and the contents of out, amax_dev, scale_dev and scale_inv_dev are undefined (blocks
+ * that gave up write nothing, blocks that got through may have written their share).  The workspace is left
+ * zeroed in that case too: the last block to leave clears it whether or not the barrier held.
  */
 fp8_status fp8_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o,
                                 uint8_t* out, float* amax_dev, float* scale_dev, float* scale_inv_dev,
@@ -137,8 +139,8 @@ size_t fp8_quantize_current_workspace_bytes(void);
  *     overlap on the GPU (different streams, or different host threads on different streams) race on
  *     it and give undefined results.  Issue them on one stream, or serialise them yourself.
  *   - n may not exceed FP8_STATIC_MAX_ELEMENTS; larger tensors return FP8_ERR_UNSUPPORTED and nothing
- *     is enqueued.  (The scratch need of this kernel does not grow with n; the bound is the largest
- *     size this entry point is exercised and supported at.)
+ *     is enqueued.  (The scratch need of this kernel does not grow with n; the bound is simply the
+ *     stated maximum of this entry point.)
  *   - Arguments, alignment rules and the bounded grid barrier are those of fp8_quantize_current.
  */
 #define FP8_STATIC_MAX_ELEMENTS ((size_t)1 << 32)
@@ -334,6 +336,24 @@ fp8_status fp8_gemm_splitk(const fp8_gemm_desc* d, const uint8_t* A, const uint8
  * so that a pipeline fault ends in an error code instead of a hung GPU.
  */
 fp8_status fp8_async_status(uint32_t* detail);
+
+/*
+ * fp8_self_test_expire_wait — the paper has no counterpart; a self-test of the library's safety net.  Every
+ * device-side wait in the library (the mbarrier waits of the GEMM pipeline, the grid barrier of
+ * fp8_quantize_current) counts SM clocks and gives up after a limit, so that a pipeline fault ends in
+ * FP8_ERR_TIMEOUT instead of a hung GPU.  This call makes one such wait run out ON PURPOSE, in a way that
+ * cannot hang or fault: it launches a small kernel whose wait can never be satisfied and whose limit is
+ * `limit_cycles` SM clocks (1 .. 2e9, i.e. at most about a second; FP8_ERR_UNSUPPORTED otherwise).
+ *   FP8_WAIT_MBARRIER      one block waits on an mbarrier nobody arrives on, through the same bounded-wait
+ *                          routine the GEMM roles use; detail code 9.
+ *   FP8_WAIT_GRID_BARRIER  the fp8_quantize_current kernel runs on an empty tensor with its grid barrier told to
+ *                          expect one block more than the grid has: every block gives up, nothing is written, the
+ *                          control words (those of fp8_quantize_current_static) are left zeroed; detail code 16.
+ * Afterwards fp8_async_status returns FP8_ERR_TIMEOUT once, with the detail code above, then FP8_OK again;
+ * the stream and the library remain fully usable.
+ */
+typedef enum { FP8_WAIT_MBARRIER = 0, FP8_WAIT_GRID_BARRIER = 1 } fp8_wait_kind;
+fp8_status fp8_self_test_expire_wait(int which, uint64_t limit_cycles, void* stream);
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* fp8_status_string(fp8_status s);

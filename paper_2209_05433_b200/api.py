@@ -25,7 +25,7 @@ EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_curr
            "fp8_scale_pow2_from_amax", "fp8_gemm", "fp8_gemm_fp8out", "fp8_amax_channels", "fp8_scales_from_amax",
            "fp8_quantize_channels", "fp8_quantize_transpose", "fp8_gemm_channel_scales", "fp8_gemm_batched",
            "fp8_gemm_splitk", "fp8_gemm_splitk_workspace",
-           "fp8_async_status", "fp8_status_string", "fp8_launch_count"]
+           "fp8_async_status", "fp8_self_test_expire_wait", "fp8_status_string", "fp8_launch_count"]
 
 
 class Fp8Error(RuntimeError):
@@ -102,6 +102,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_gemm_splitk.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.fp8_async_status.restype = i32
     lib.fp8_async_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
+    lib.fp8_self_test_expire_wait.restype = i32
+    lib.fp8_self_test_expire_wait.argtypes = [i32, ctypes.c_uint64, vp]
     lib.fp8_status_string.restype = ctypes.c_char_p
     lib.fp8_status_string.argtypes = [i32]
     lib.fp8_launch_count.restype = ctypes.c_uint64
@@ -393,11 +395,26 @@ def fp8_gemm_batched(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int
                                    None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()), "fp8_gemm_batched")
 
 
+TIMEOUT = 7                                   # FP8_ERR_TIMEOUT
+WAIT_MBARRIER, WAIT_GRID_BARRIER = 0, 1       # fp8_wait_kind
+
+
 def fp8_async_status() -> tuple[int, int]:
-    """(status, detail) of the device-side error latch; synchronises the device."""
+    """(status, detail) of the device-side error latch; synchronises the device.  After a time-out the cached
+    current-scaling workspaces are cleared again (the kernel leaves them zeroed; this costs nothing and does not
+    rely on it)."""
     detail = ctypes.c_uint32(0)
     s = load().fp8_async_status(ctypes.byref(detail))
+    if int(s) == TIMEOUT:
+        for ws in _workspaces.values():
+            ws.zero_()
+        torch.cuda.synchronize()
     return int(s), int(detail.value)
+
+
+def fp8_self_test_expire_wait(which: int, limit_cycles: int = 2_000_000) -> None:
+    """Makes one bounded device-side wait run out on purpose (about a millisecond by default); see the header."""
+    _check(load().fp8_self_test_expire_wait(which, limit_cycles, _stream()), "fp8_self_test_expire_wait")
 
 
 def fp8_launch_count() -> int:

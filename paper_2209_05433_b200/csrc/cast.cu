@@ -23,6 +23,7 @@ void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order
 
 fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o, uint8_t* out,
                                    float* amax, float* scale, float* scale_inv, unsigned int* ws, cudaStream_t st);
+fp8_status launch_grid_barrier_self_test(long long limit_cycles, cudaStream_t st);
 
 int sm_count() {
     static std::mutex mu;
@@ -40,68 +41,16 @@ int sm_count() {
 
 constexpr int kWideF32 = 0;
 constexpr int kWideBF16 = 1;
-#ifndef FP8_CAST_THREADS
-#define FP8_CAST_THREADS 256
-#endif
-#ifndef FP8_QUANT_UNROLL_BF16
-#define FP8_QUANT_UNROLL_BF16 2
-#endif
-#ifndef FP8_DEQUANT_UNROLL
-#define FP8_DEQUANT_UNROLL 4
-#endif
-#ifndef FP8_AMAX_UNROLL
-#define FP8_AMAX_UNROLL 8
-#endif
-constexpr int kThreads = FP8_CAST_THREADS;
+constexpr int kThreads = 256;
 
-// Input loads of the streaming kernels: read-only path without L1 allocation.  Plain loads (FP8_PLAIN_LOADS) were
-// measured too: faster on tensors far larger than L2 (amax +4 %, quantize +2.5 %, binary32-input quantize +7 %) but
-// slower whenever part of the tensor sits in L2 (2^24 elements: amax 2950 -> 2194 GB/s; per-column kernels -6..-15 %)
-// and 2 % slower for the casts inside the benchmark step, so they are not the default.
-__device__ __forceinline__ uint4 ld_in_v4(const void* p) {
-#ifdef FP8_PLAIN_LOADS
-    return *reinterpret_cast<const uint4*>(p);
-#else
-    return ld_nc_v4(p);
-#endif
-}
-__device__ __forceinline__ uint2 ld_in_v2(const void* p) {
-#ifdef FP8_PLAIN_LOADS
-    return *reinterpret_cast<const uint2*>(p);
-#else
-    return ld_nc_v2(p);
-#endif
-}
+// Input loads of the streaming kernels take the read-only path without L1 allocation (plain loads are a few
+// per cent faster on tensors far larger than L2 but slower whenever part of the tensor sits in L2).
+__device__ __forceinline__ uint4 ld_in_v4(const void* p) { return ld_nc_v4(p); }
+__device__ __forceinline__ uint2 ld_in_v2(const void* p) { return ld_nc_v2(p); }
 
-// Output stores: written once, never re-read by the same kernel.
-__device__ __forceinline__ void st_out(uint2* p, uint2 v) {
-#ifdef FP8_STORE_CS
-    __stcs(p, v);
-#else
-    *p = v;
-#endif
-}
-__device__ __forceinline__ void st_out(uint32_t* p, uint32_t v) {
-#ifdef FP8_STORE_CS
-    __stcs(p, v);
-#else
-    *p = v;
-#endif
-}
-__device__ __forceinline__ void st_out(uint4* p, uint4 v) {
-#ifdef FP8_STORE_CS
-    __stcs(p, v);
-#else
-    *p = v;
-#endif
-}
-__device__ __forceinline__ void st_out(float4* p, float4 v) {
-#ifdef FP8_STORE_CS
-    __stcs(p, v);
-#else
-    *p = v;
-#endif
-}
+// Output stores: written once, never re-read by the same kernel; default write-back policy.
+template <typename T>
+__device__ __forceinline__ void st_out(T* p, T v) { *p = v; }
 
 // ---------------------------------------------------------------------------
 // per-item arithmetic
@@ -411,19 +360,10 @@ __device__ unsigned int g_cast_latch[2] = {0u, 0u};
 constexpr unsigned int kWaitGridBarrier = 16u;
 constexpr long long kGridWaitLimitCycles = 4000000000ll;       // about 2 s of SM clocks
 
-// One-launch current scaling: megabytes of the end of x asked to stay in L2 between the passes, for tensors
-// larger than FP8_CURRENT_KEEP_FROM_MB (smaller ones are left to the default replacement: they mostly fit).
-// Measured together with plain second-pass loads over a ring of distinct 2^28-element bf16 tensors: 6.35 -> 6.67 TB/s
-// (repeated calls on one tensor gain more, but only because the second pass ends where the next first pass starts).
-#ifndef FP8_CURRENT_KEEP_MB
-#define FP8_CURRENT_KEEP_MB 96
-#endif
-#ifndef FP8_CURRENT_KEEP_FROM_MB
-#define FP8_CURRENT_KEEP_FROM_MB 160
-#endif
-#ifndef FP8_CURRENT_PLAIN_REREAD
-#define FP8_CURRENT_PLAIN_REREAD 1
-#endif
+// One-launch current scaling of a tensor larger than kCurrentKeepFromMB: the last kCurrentKeepMB megabytes read by
+// the first pass are asked to stay in L2 (the second pass starts there), the rest to leave first.  Smaller tensors
+// are left to the default replacement: they mostly fit.
+constexpr size_t kCurrentKeepMB = 96, kCurrentKeepFromMB = 160;
 __device__ __forceinline__ uint64_t l2_policy_evict_last() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
@@ -447,10 +387,13 @@ __device__ __forceinline__ uint4 ld_v4_policy(const void* ptr, uint64_t policy) 
 // grid barrier, ws[2] = departures; the three words are zero on entry and the last CTA to leave puts
 // them back to zero.  The second pass walks each CTA's chunks in reverse so that the part of x read
 // last in the first pass is re-read from L2.
+// `arrivals` is the number of CTAs the barrier waits for (the grid size; the wait self-test passes one more, which
+// can never arrive) and `wait_limit` the SM clocks a CTA waits before it gives up.
 template <int WIDE, int FMT, bool NOSAT, int UNROLL>
 __global__ void __launch_bounds__(kThreads)
 k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __restrict__ out,
-                   float* amax_out, float* scale_out, float* scale_inv_out, unsigned int* ws) {
+                   float* amax_out, float* scale_out, float* scale_inv_out, unsigned int* ws,
+                   unsigned int arrivals, long long wait_limit) {
     __shared__ uint32_t red[32];
     __shared__ uint32_t bcast[2];
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
@@ -461,11 +404,9 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
     const size_t tail = n - n_items * EPI;
 
     // ---- pass 1: amax
-    // a large tensor: its last FP8_CURRENT_KEEP_MB megabytes are asked to stay in L2 for the second pass (which
-    // starts there), the rest to leave first; a small one: default replacement
-    const bool large = FP8_CURRENT_KEEP_MB > 0 && n_chunks * per_chunk * 16 > ((size_t)FP8_CURRENT_KEEP_FROM_MB << 20);
+    const bool large = n_chunks * per_chunk * 16 > (kCurrentKeepFromMB << 20);
     const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
-    const size_t keep_chunks = ((size_t)FP8_CURRENT_KEEP_MB << 20) / (per_chunk * 16);
+    const size_t keep_chunks = (kCurrentKeepMB << 20) / (per_chunk * 16);
     const size_t keep_from = n_chunks > keep_chunks ? n_chunks - keep_chunks : 0;
     uint32_t m = 0;
     for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
@@ -501,11 +442,11 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
         for (uint32_t spins = 1;; ++spins) {
             unsigned int arrived;
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(arrived) : "l"(&ws[1]) : "memory");
-            if (arrived >= gridDim.x) break;
+            if (arrived >= arrivals) break;
             if ((spins & 255u) == 0u) {
                 const long long now = clock64();
                 if (t0 == 0) t0 = now;
-                else if (now - t0 > kGridWaitLimitCycles) {
+                else if (now - t0 > wait_limit) {
                     if (atomicCAS(&g_cast_latch[0], 0u, kWaitGridBarrier) == 0u) g_cast_latch[1] = blockIdx.x;
                     okflag = 0u;
                     break;
@@ -537,11 +478,7 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
             if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
                 uint4 v[UNROLL];
 #pragma unroll
-#if FP8_CURRENT_PLAIN_REREAD
-                for (int u = 0; u < UNROLL; ++u) v[u] = *(xv + base + (size_t)u * kThreads);
-#else
-                for (int u = 0; u < UNROLL; ++u) v[u] = ld_nc_v4(xv + base + (size_t)u * kThreads);
-#endif
+                for (int u = 0; u < UNROLL; ++u) v[u] = *(xv + base + (size_t)u * kThreads);      // plain loads: the re-read hits L2
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) {
                     const size_t i = base + (size_t)u * kThreads;
@@ -678,9 +615,7 @@ __global__ void k_scale_pow2_from_amax(const float* amax_dev, float fmax, float*
 // (8 bf16 / 4 f32) and every fourth row of the block's slab; per-column maxima stay separate inside the
 // packed words.  The four row lanes meet in shared memory, then one atomicMax per column per block.
 // amax_bits[cols] must be zero before.
-#ifndef FP8_COLS_MIN_ROWS
-#define FP8_COLS_MIN_ROWS 256
-#endif
+constexpr int kColsMinRows = 256;
 constexpr int kColsTx = 64, kColsTy = 4, kColsUnroll = 8;       // 64 x 4 threads, eight row loads in flight per thread
 template <int WIDE>
 __global__ void __launch_bounds__(kColsTx * kColsTy)
@@ -951,19 +886,10 @@ __device__ __forceinline__ void transpose_4x4_bytes(uint32_t a0, uint32_t a1, ui
     t[3] = __byte_perm(hi01, hi23, 0x7632);
 }
 
-#ifndef FP8_TR_MIN_CTAS_BF16
-#define FP8_TR_MIN_CTAS_BF16 4
-#endif
-#ifndef FP8_TR_MIN_CTAS_F32
-#define FP8_TR_MIN_CTAS_F32 3
-#endif
-#ifndef FP8_TR_THREADS_F32
-#define FP8_TR_THREADS_F32 256
-#endif
-// threads per CTA and CTAs per SM (measured best: 4 x 256 threads for bf16 input, 3 x 256 for binary32)
+// threads per CTA and CTAs per SM: 4 x 256 threads for bf16 input, 3 x 256 for binary32
 template <int WIDE> struct TrGeo {
-    static constexpr int THREADS = WIDE == kWideBF16 ? kThreads : FP8_TR_THREADS_F32;
-    static constexpr int MIN_CTAS = WIDE == kWideBF16 ? FP8_TR_MIN_CTAS_BF16 : FP8_TR_MIN_CTAS_F32;
+    static constexpr int THREADS = kThreads;
+    static constexpr int MIN_CTAS = WIDE == kWideBF16 ? 4 : 3;
 };
 
 // One 128 x 128 tile per CTA, 8 or 16 warps, several CTAs resident per SM (the loads in flight live in registers, so
@@ -1074,21 +1000,10 @@ k_quantize_transpose_elementwise(const void* __restrict__ x, int64_t rows, int64
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Persistent grid: enough blocks to fill every SM (at most `per_sm_cap` of them per SM), no more than there is work.
-// Kernels that mix a read and a write stream run faster with fewer resident CTAs than fit (measured, bf16 input,
-// 2^29 elements: quantize 6.11 -> 6.37 TB/s at 6 per SM, dequantize 5.65 -> 5.97 at 3, the simulated round trip
-// 5.88 -> 6.18 at 5); the read-only amax and the two-pass current scaling are fastest at full residency.
-#ifndef FP8_QUANT_PER_SM
-#define FP8_QUANT_PER_SM 6
-#endif
-#ifndef FP8_DEQUANT_PER_SM
-#define FP8_DEQUANT_PER_SM 3
-#endif
-#ifndef FP8_FAKE_PER_SM
-#define FP8_FAKE_PER_SM 5
-#endif
-#ifndef FP8_CURRENT_PER_SM
-#define FP8_CURRENT_PER_SM 64
-#endif
+// Kernels that mix a read and a write stream run faster with fewer resident CTAs than fit: quantize 6 per SM,
+// dequantize 3, the simulated round trip 5 (4-6 % over full residency on 2^29 bf16 elements); the read-only amax and
+// the two-pass current scaling are fastest at full residency.
+constexpr int kQuantPerSM = 6, kDequantPerSM = 3, kFakePerSM = 5, kCurrentPerSM = 64;
 template <typename Kernel>
 static int persistent_grid(Kernel kernel, size_t work_chunks, int per_sm_cap = 64) {
     int per_sm = 0;
@@ -1107,10 +1022,11 @@ static size_t chunks_of(size_t n, int epi, int unroll) {
     return (items + per_chunk - 1) / per_chunk;
 }
 
-constexpr int kAmaxUnroll = FP8_AMAX_UNROLL;
-constexpr int kQuantUnrollBF16 = FP8_QUANT_UNROLL_BF16;
+// independent 16-byte loads in flight per thread
+constexpr int kAmaxUnroll = 8;
+constexpr int kQuantUnrollBF16 = 2;
 constexpr int kQuantUnrollF32 = 8;
-constexpr int kDequantUnroll = FP8_DEQUANT_UNROLL;
+constexpr int kDequantUnroll = 4;
 
 template <int WIDE>
 static fp8_status launch_amax(const void* x, size_t n, uint32_t* bits, cudaStream_t st) {
@@ -1134,7 +1050,7 @@ static fp8_status launch_quantize(const void* x, size_t n, const float* scale, u
     // the vector path stores EPI codes per item: out must be EPI-byte aligned, x 16-byte aligned
     if (aligned16(x) && (reinterpret_cast<uintptr_t>(out) & (EPI - 1)) == 0) {
         auto k = k_quantize<WIDE, FMT, NOSAT, WITH_AMAX, UNROLL>;
-        const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL), FP8_QUANT_PER_SM);
+        const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL), kQuantPerSM);
         k<<<grid, kThreads, 0, st>>>(x, n, scale, out, bits);
     } else {
         auto k = k_quantize_elementwise<WIDE, FMT, NOSAT, WITH_AMAX>;
@@ -1158,7 +1074,7 @@ static fp8_status launch_dequantize(const uint8_t* c, size_t n, const float* si,
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
     if (aligned16(out) && (reinterpret_cast<uintptr_t>(c) & (EPI - 1)) == 0) {
         auto k = k_dequantize<FMT, WIDE, kDequantUnroll>;
-        const int grid = persistent_grid(k, chunks_of(n, EPI, kDequantUnroll), FP8_DEQUANT_PER_SM);
+        const int grid = persistent_grid(k, chunks_of(n, EPI, kDequantUnroll), kDequantPerSM);
         k<<<grid, kThreads, 0, st>>>(c, n, si, out);
     } else {
         auto k = k_dequantize_elementwise<FMT, WIDE>;
@@ -1183,8 +1099,11 @@ static fp8_status launch_current(const void* x, size_t n, float fmax, uint8_t* o
     auto k = k_quantize_current<WIDE, FMT, NOSAT, UNROLL>;
     size_t chunks = chunks_of(n, EPI, UNROLL);
     if (chunks < 1) chunks = 1;
-    const int grid = persistent_grid(k, chunks, FP8_CURRENT_PER_SM);   // co-resident by construction: SMs x occupancy at most
-    void* args[] = {(void*)&x, (void*)&n, (void*)&fmax, (void*)&out, (void*)&amax, (void*)&scale, (void*)&scale_inv, (void*)&ws};
+    const int grid = persistent_grid(k, chunks, kCurrentPerSM);   // co-resident by construction: SMs x occupancy at most
+    unsigned int arrivals = (unsigned int)grid;
+    long long wait_limit = kGridWaitLimitCycles;
+    void* args[] = {(void*)&x, (void*)&n, (void*)&fmax, (void*)&out, (void*)&amax, (void*)&scale, (void*)&scale_inv, (void*)&ws,
+                    (void*)&arrivals, (void*)&wait_limit};
     if (cudaLaunchCooperativeKernel((const void*)k, dim3(grid), dim3(kThreads), args, 0, st) != cudaSuccess) {
         (void)cudaGetLastError();                                  // e.g. the device cannot hold the whole grid right now
         return FP8_ERR_UNSUPPORTED;                                // the caller falls back to the three separate kernels
@@ -1232,7 +1151,7 @@ static fp8_status launch_fake(const void* x, size_t n, const float* scale, const
     constexpr int UNROLL = 2;
     if (aligned16(x) && aligned16(out)) {
         auto k = k_fake_quantize<WIDE, FMT, NOSAT, UNROLL>;
-        const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL), FP8_FAKE_PER_SM);
+        const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL), kFakePerSM);
         k<<<grid, kThreads, 0, st>>>(x, n, scale, si, out);
     } else {
         auto k = k_fake_quantize_elementwise<WIDE, FMT, NOSAT>;
@@ -1265,7 +1184,7 @@ static int64_t slab_rows(int64_t rows, int64_t col_blocks) {
     if (slabs < 1) slabs = 1;
     int64_t per = (rows + slabs - 1) / slabs;
     per = (per + 15) / 16 * 16;
-    if (per < FP8_COLS_MIN_ROWS) per = FP8_COLS_MIN_ROWS;          // short slabs are all launch, tail and atomics
+    if (per < kColsMinRows) per = kColsMinRows;          // short slabs are all launch, tail and atomics
     while ((rows + per - 1) / per > 65535) per *= 2;
     return per;
 }
@@ -1605,3 +1524,30 @@ const char* fp8_status_string(fp8_status s) {
 uint64_t fp8_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"
+
+// Self-test of the bounded grid barrier: the one-launch kernel on an empty tensor, its barrier told to wait for one
+// CTA more than the grid has.  Every CTA gives up after `limit_cycles`, latches the time-out and returns without
+// writing anything; the last one out leaves the control words zeroed, as always.  Uses the static control words.
+fp8_status fp8b200::launch_grid_barrier_self_test(long long limit_cycles, cudaStream_t st) {
+    unsigned int* scratch = nullptr;
+    fp8_status s = static_scratch_address(&scratch);
+    if (s != FP8_OK) return s;
+    if (cudaMemsetAsync(scratch, 0, 16, st) != cudaSuccess) return FP8_ERR_CUDA;
+    count_launches(1);
+    auto k = k_quantize_current<kWideBF16, kE4M3, false, 4>;
+    const void* x = nullptr;
+    size_t n = 0;
+    float fmax = 448.0f;
+    uint8_t* out = nullptr;
+    float* none = nullptr;
+    const int grid = 8;
+    unsigned int arrivals = (unsigned int)grid + 1u;
+    void* args[] = {(void*)&x, (void*)&n, (void*)&fmax, (void*)&out, (void*)&none, (void*)&none, (void*)&none, (void*)&scratch,
+                    (void*)&arrivals, (void*)&limit_cycles};
+    if (cudaLaunchCooperativeKernel((const void*)k, dim3(grid), dim3(kThreads), args, 0, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return FP8_ERR_CUDA;
+    }
+    count_launches(1);
+    return launch_status();
+}

@@ -38,11 +38,6 @@ __device__ __forceinline__ uint2 ld_nc_v2(const void* p) {
 
 __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
     uint4 v;
-#ifdef FP8_LOAD_L2_256B
-    asm volatile("ld.global.nc.L1::no_allocate.L2::256B.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-#endif
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;

@@ -29,8 +29,6 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include <cstdio>
-#include <cstdlib>
 #include <mutex>
 
 #include "codec.cuh"
@@ -42,19 +40,6 @@ __device__ unsigned int g_async_latch[2] = {0u, 0u};
 
 namespace gemm {
 
-#ifdef FP8_GEMM_PROFILE
-// Development aid, absent from the product build: per-CTA cycle counters of where each role waits.
-__device__ unsigned long long g_prof[512 * 8];
-#define PROF_DECL long long prof_t = 0, prof_acc0 = 0, prof_acc1 = 0; const long long prof_start = clock64();
-#define PROF_BEGIN prof_t = clock64();
-#define PROF_END(acc) acc += clock64() - prof_t;
-#define PROF_STORE(slot0, slot1, slot2) if (lane == 0) { g_prof[blockIdx.x * 8 + slot0] = prof_acc0; g_prof[blockIdx.x * 8 + slot1] = prof_acc1; if (slot2 >= 0) g_prof[blockIdx.x * 8 + slot2] = clock64() - prof_start; }
-#else
-#define PROF_DECL
-#define PROF_BEGIN
-#define PROF_END(acc)
-#define PROF_STORE(slot0, slot1, slot2)
-#endif
 
 constexpr int BM = 128;             // tile rows  (= UMMA M, one TMEM lane per row)
 constexpr int BN = 256;             // tile cols  (= UMMA N, one TMEM column per col)
@@ -88,7 +73,7 @@ constexpr int GROUP_M = 16;         // tile raster: GROUP_M row-tiles share each
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clocks per wait
 
 // codes written to the error latch
-enum : uint32_t { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC_EMPTY = 3, WAIT_ACC_FULL = 4 };
+enum : uint32_t { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC_EMPTY = 3, WAIT_ACC_FULL = 4, WAIT_SELF_TEST = 9 };
 
 // ---- PTX wrappers ----------------------------------------------------------
 
@@ -112,10 +97,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false after about WAIT_LIMIT_CYCLES SM clocks (checked every 1024 failed
-// polls, so that the common short wait never reads a timer), or as soon as another role of this CTA
-// has given up (abort flag), having latched `code`.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code) {
+// Bounded wait.  Returns false after about `limit` SM clocks (checked every 1024 failed polls, so that
+// the common short wait never reads a timer), or as soon as another role of this CTA has given up
+// (abort flag), having latched `code`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code,
+                                          long long limit = WAIT_LIMIT_CYCLES) {
     long long t0 = 0;
     for (uint32_t spins = 1;; ++spins) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -123,7 +109,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_CYCLES) {
+            else if (now - t0 > limit) {
                 *abort_flag = 1u;
                 if (atomicCAS(&g_async_latch[0], 0u, code) == 0u) g_async_latch[1] = blockIdx.x;
                 return false;
@@ -391,7 +377,6 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         const uint64_t keep = policy_evict_last();
-        PROF_DECL
         for (int t = worker; t < num_tiles && ok; t += num_workers) {
             int tm, tn;
             const int bi = t / tiles_per_batch;                                 // batch member
@@ -399,9 +384,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             const int m0 = tm * G::TILE_M + (int)cta_rank * BM;                 // this CTA's 128 rows of A
             const int n0 = tn * BN + (int)cta_rank * (BN / CG);                 // this CTA's rows of B
             for (int kb = 0; kb < k_pad; ++kb) {
-                PROF_BEGIN
                 ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, WAIT_EMPTY);
-                PROF_END(prof_acc0)
                 if (!ok) break;
                 if (lane == 0) {
                     const uint32_t sa = ring + stage * STAGE_BYTES;
@@ -439,7 +422,6 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-        PROF_STORE(0, 1, 2)
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         uint32_t stage = 0, phase = 0;
@@ -447,13 +429,10 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         int it = 0;
         const uint32_t a_kstep = A_MN ? UMMA_K * 128 : UMMA_K, a_lbo = A_MN ? BK * 128 : 16;
         const uint32_t b_kstep = B_MN ? UMMA_K * 128 : UMMA_K, b_lbo = B_MN ? BK * 128 : 16;
-        PROF_DECL
         for (int t = worker; t < num_tiles && ok; t += num_workers) {
           for (int kc = 0; kc < k_pad && ok; kc += chunk_blocks, ++it) {          // `it` counts accumulator uses
             const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
-            PROF_BEGIN
             ok = mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag, WAIT_ACC_EMPTY);
-            PROF_END(prof_acc1)
             if (!ok) break;
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * BN;
@@ -461,9 +440,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             const int last_real = min(k_blocks, kend) - 1;                        // its MMAs complete the accumulator
             for (int kb = kc; kb < kend; kb += FG) {
                 // one wait per TWO K-blocks: every barrier query between MMA issues costs about one MMA time
-                PROF_BEGIN
                 ok = mbar_wait(smem_u32(&bars->full[stage / FG]), phase, abort_flag, WAIT_FULL);
-                PROF_END(prof_acc0)
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
@@ -500,7 +477,6 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             }
           }
         }
-        PROF_STORE(3, 4, 5)
     } else {
         // ------------------------------------------------------------ epilogue (each CTA drains its own 128 rows)
         const int q = warp & 3;                                   // TMEM lane quarter this warp may read
@@ -516,7 +492,6 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         const uint64_t stream_out = policy_evict_first();
         bool ok = true;
         int it = 0;
-        PROF_DECL
         float part[SPLIT ? 128 : 1];                              // split accumulation: this thread's 128 partial sums
         for (int t = worker; t < num_tiles && ok; t += num_workers) {
           int tm, tn;
@@ -524,9 +499,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
           tile_coords(t - bi * tiles_per_batch, p.tiles_m, p.tiles_n, tm, tn);
           for (int kc = 0; kc < k_pad && ok; kc += chunk_blocks, ++it) {         // `it` counts accumulator uses
             const uint32_t acc = (uint32_t)it & 1u, acc_phase = ((uint32_t)it >> 1) & 1u;
-            PROF_BEGIN
             ok = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, WAIT_ACC_FULL);
-            PROF_END(prof_acc0)
             if (!ok) break;
             tc_fence_after();
             const int row0 = tm * G::TILE_M + (int)cta_rank * BM + q * 32;      // first of this warp's 32 rows
@@ -669,7 +642,6 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
           }
         }
         if (lane == 0) bulk_wait_all();                           // every store has reached global memory before exit
-        if (warp == 2) { PROF_STORE(6, 7, -1) }
         if (p.amax_bits) {
             uint32_t bits = OUT == OUT_BF16 ? (max(running & 0xFFFFu, running >> 16) << 16) : __float_as_uint(runf);
             bits = warp_max_u32(canonical_nan_bits(bits));
@@ -722,12 +694,15 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
 }
 
 // CTA-pair kernels launch as clusters of 2; the grid is one CTA per SM that can be paired.
+// The dynamic shared-memory attribute and the number of co-resident clusters are properties of
+// (kernel instance, device): looked up on the first launch of an instance on a device, then reused.
 template <int CG, int OUT, int EPI_WARPS, bool SPLIT = false>
 static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const Params& p, int64_t num_tiles, cudaStream_t st) {
     auto k = k_gemm_fp8<CG, OUT, EPI_WARPS, SPLIT>;
     constexpr int THREADS = 64 + 32 * EPI_WARPS;
-    // per device and cheap, so set on every launch rather than cached
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return FP8_ERR_CUDA;
+    constexpr int MAX_DEVICES = 64;
+    static std::mutex mu;
+    static int cached_workers[MAX_DEVICES] = {0};                 // 0 = not looked up yet
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(THREADS, 1, 1);
     cfg.dynamicSmemBytes = SMEM_BYTES;
@@ -739,15 +714,25 @@ static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUt
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    int workers = sm_count() / CG;
-    if (CG == 2) {
-        cfg.gridDim = dim3(2 * workers, 1, 1);
-        int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, k, &cfg) == cudaSuccess && clusters > 0 && clusters < workers) workers = clusters;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FP8_ERR_CUDA;
+    int workers = 0;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (dev >= 0 && dev < MAX_DEVICES) workers = cached_workers[dev];
+        if (workers == 0) {
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return FP8_ERR_CUDA;
+            workers = sm_count() / CG;
+            if (CG == 2) {
+                cfg.gridDim = dim3(2 * workers, 1, 1);
+                int clusters = 0;
+                if (cudaOccupancyMaxActiveClusters(&clusters, k, &cfg) == cudaSuccess && clusters > 0 && clusters < workers) workers = clusters;
+            }
+            if (dev >= 0 && dev < MAX_DEVICES) cached_workers[dev] = workers;
+        }
     }
     if ((int64_t)workers > num_tiles) workers = (int)num_tiles;
     cfg.gridDim = dim3(workers * CG, 1, 1);
-    if (getenv("FP8_B200_DEBUG")) fprintf(stderr, "[fp8_b200] gemm CG=%d grid=%d tiles=%lld\n", CG, workers * CG, (long long)num_tiles);
     if (cudaLaunchKernelEx(&cfg, k, ma, mb, md, p) != cudaSuccess) return FP8_ERR_CUDA;
     count_launches(1);
     return launch_status();
@@ -935,7 +920,25 @@ static int choose_splits(int64_t M, int64_t N, int64_t K) {
     return best_t <= 0.85 * base ? best : 1;
 }
 
+// Self-test of the bounded mbarrier wait: one CTA initialises a barrier that nobody arrives on and waits
+// for it with the given limit; the wait gives up, latches WAIT_SELF_TEST and the kernel returns.
+__global__ void k_wait_self_test(long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0u;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) (void)mbar_wait(smem_u32(&bar), 0u, &abort_flag, WAIT_SELF_TEST, limit_cycles);
+    __syncthreads();
+}
+
 }  // namespace gemm
+
+fp8_status launch_grid_barrier_self_test(long long limit_cycles, cudaStream_t st);      // defined with the cast kernels
+
 }  // namespace fp8b200
 
 using namespace fp8b200;
@@ -1042,12 +1045,16 @@ fp8_status fp8_gemm_splitk(const fp8_gemm_desc* d, const uint8_t* A, const uint8
     return launch_status();
 }
 
-#ifdef FP8_GEMM_PROFILE
-int fp8_debug_gemm_profile(unsigned long long* host_out, int n) {
-    cudaDeviceSynchronize();
-    return (int)cudaMemcpyFromSymbol(host_out, fp8b200::gemm::g_prof, sizeof(unsigned long long) * n);
+
+fp8_status fp8_self_test_expire_wait(int which, uint64_t limit_cycles, void* stream) {
+    if (which != FP8_WAIT_MBARRIER && which != FP8_WAIT_GRID_BARRIER) return FP8_ERR_ENUM;
+    if (limit_cycles == 0 || limit_cycles > 2000000000ull) return FP8_ERR_UNSUPPORTED;      // at most about a second
+    cudaStream_t st = (cudaStream_t)stream;
+    if (which == FP8_WAIT_GRID_BARRIER) return fp8b200::launch_grid_barrier_self_test((long long)limit_cycles, st);
+    fp8b200::gemm::k_wait_self_test<<<1, 32, 0, st>>>((long long)limit_cycles);
+    count_launches(1);
+    return launch_status();
 }
-#endif
 
 void fp8_cast_read_clear_latch(unsigned int out2[2]);      // defined with the cast kernels
 

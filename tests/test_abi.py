@@ -12,6 +12,25 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 HEADER = os.path.join(ROOT, "include", "fp8_b200.h")
 
 
+_keep = []
+
+
+def _addresses():
+    """(an aligned address, one that is not 16-byte aligned) for the argument-error calls.  Every such call fails
+    validation before anything is enqueued, so the addresses are never dereferenced; on a machine with a GPU they
+    still point into a real device buffer, so that even a library bug that enqueued work could not touch memory
+    this process does not own."""
+    try:
+        import torch
+        if torch.cuda.is_available():
+            buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+            _keep.append(buf)
+            return ctypes.c_void_p(buf.data_ptr()), ctypes.c_void_p(buf.data_ptr() + 8)
+    except Exception:
+        pass
+    return ctypes.c_void_p(16), ctypes.c_void_p(24)
+
+
 def _declared():
     text = open(HEADER).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
@@ -35,7 +54,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_argument_errors_are_reported_before_any_launch():
     lib = api.load()
-    one = ctypes.c_void_p(16)          # never dereferenced: every call below fails validation first
+    one, odd = _addresses()            # never dereferenced: every call below fails validation first
     assert lib.fp8_amax(one, 0, 4, None, None) == 1                      # FP8_ERR_NULL
     assert lib.fp8_amax(one, 7, 4, one, None) == 2                       # FP8_ERR_ENUM
     assert lib.fp8_scale_from_amax(None, 0, one, one, None) == 1
@@ -62,19 +81,19 @@ def test_argument_errors_are_reported_before_any_launch():
     d.lda = 136                                                                         # not a multiple of 16
     assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 4       # FP8_ERR_ALIGN
     d.lda = 128
-    assert lib.fp8_gemm(ctypes.byref(d), ctypes.c_void_p(24), one, one, one, one, None, None) == 4
+    assert lib.fp8_gemm(ctypes.byref(d), odd, one, one, one, one, None, None) == 4
     d.ldd = 100                                                                         # smaller than N
     assert lib.fp8_gemm(ctypes.byref(d), one, one, one, one, one, None, None) == 3
 
 
 def test_argument_errors_of_the_wider_entry_points():
     lib = api.load()
-    one = ctypes.c_void_p(16)
+    one, odd = _addresses()
     # one-launch current scaling: null pointers, enums, workspace alignment
     assert lib.fp8_quantize_current(one, 1, 4, 0, 0, one, None, one, one, one, None) == 1
     assert lib.fp8_quantize_current(one, 1, 4, 0, 0, one, one, one, one, None, None) == 1
     assert lib.fp8_quantize_current(one, 1, 4, 5, 0, one, one, one, one, one, None) == 2
-    assert lib.fp8_quantize_current(one, 1, 4, 0, 0, one, one, one, one, ctypes.c_void_p(24), None) == 4
+    assert lib.fp8_quantize_current(one, 1, 4, 0, 0, one, one, one, one, odd, None) == 4
     assert lib.fp8_quantize_current_workspace_bytes() == 16
     assert lib.fp8_quantize_current_static(one, 1, 4, 0, 0, one, None, one, one, None) == 1
     assert lib.fp8_quantize_current_static(one, 9, 4, 0, 0, one, one, one, one, None) == 2

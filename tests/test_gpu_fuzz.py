@@ -104,7 +104,7 @@ def test_random_fp8_output_case(seed):
     assert api.fp8_async_status()[0] == 0
     assert bool((D_full[M:, :] == 0xA5).all()) and bool((D_full[:M, N:] == 0xA5).all()), "wrote outside D"
     enc = lambda y: oracle.quantize(y.reshape(-1), 1.0, fd, overflow).reshape(y.shape)
-    ok = check_gemm_fp8out(D.cpu().numpy(), ref, sabs, scale_d, enc)
+    ok, _ = check_gemm_fp8out(D.cpu().numpy(), ref, sabs, scale_d, enc)
     assert ok.all(), ((M, N, K, fa, fb, fd, ma, mb, acc, overflow), np.argwhere(~ok)[:4].tolist())
     lo = np.max(np.abs(ref) - 1e-5 * sabs) * (1 - 2.0 ** -22)
     hi = np.max(np.abs(ref) + 1e-5 * sabs) * (1 + 2.0 ** -22)

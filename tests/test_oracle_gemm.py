@@ -139,3 +139,69 @@ def test_per_channel_scales_reduce_to_per_tensor_routines():
     for j in range(N):
         r1, s1 = oracle.gemm_rows(A, E4M3, (K, 1), B, E4M3, (N, 1), N, K, 0, M, 0.5, sv[j])
         assert np.array_equal(ref[:, j], r1[:, j]) and np.array_equal(sab[:, j], s1[:, j])
+
+
+def _nearest_code(y32, fmt):
+    """Saturating round-to-nearest-even by exhaustive search over the decode table (reads only the table,
+    pinned separately against Table 1): the lowest code among the nearest magnitudes, moved up one when the
+    next magnitude is equally near and the found one is odd; beyond the midpoint past the maximum, the maximum."""
+    t = oracle.decode_table(fmt)
+    maxmag = 0x7E if fmt == E4M3 else 0x7B
+    ext = np.concatenate([t[: maxmag + 1], [480.0 if fmt == E4M3 else 65536.0]])
+    a = np.abs(y32.astype(np.float64)).reshape(-1)
+    d = np.abs(a[:, None] - ext[None, :])
+    best = np.argmin(d, axis=1)
+    nxt = np.minimum(best + 1, ext.size - 1)
+    rows = np.arange(a.size)
+    tie = (d[rows, nxt] == d[rows, best]) & (nxt != best)
+    best = np.where(tie & (best % 2 == 1), nxt, best)
+    best = np.minimum(best, maxmag)
+    sign = ((y32.reshape(-1).view(np.uint32) >> 31) << 7).astype(np.uint8)
+    return (sign | best.astype(np.uint8)).reshape(y32.shape)
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2])
+def test_per_channel_routines_equal_numpy_closed_forms(fmt):
+    """Section 4.2, per-channel scales, against definitions written with numpy alone: the per-channel amax is
+    np.abs(x).max along the other axis; the codes are the nearest-code search applied to x * s broadcast along
+    the channel axis (one binary32 multiply); the column-scaled product is the plain float64 matmul of the
+    decoded operands times sa_inv * sb_inv[j].  A row/column mix-up, a wrong pitch or a scale applied along the
+    wrong axis fails here on the non-square shapes."""
+    rng = np.random.default_rng(77 + fmt)
+    rows, cols = 29, 45
+    x = (rng.standard_normal((rows, cols)) * np.exp2(rng.uniform(-5, 5, size=(rows, cols)))).astype(np.float32)
+    x[:, 3] *= 64.0                                  # a column and a row that dominate their channels
+    x[11, :] *= 32.0
+    for axis in (0, 1):
+        am = oracle.amax_channels(x, axis)
+        assert am.shape == ((cols,) if axis == 0 else (rows,))
+        assert np.array_equal(am, np.abs(x).max(axis=axis))
+        s = (np.float32(oracle.FMT_MAX[fmt]) / am).astype(np.float32)
+        y = x * (s[None, :] if axis == 0 else s[:, None])          # binary32 multiply, broadcast along the channel axis
+        assert np.array_equal(oracle.quantize_channels(x, s, axis, fmt), _nearest_code(y, fmt))
+        # the same through bf16 inputs (exact widening)
+        xb = (x.view(np.uint32) >> 16).astype(np.uint16)
+        xw = (xb.astype(np.uint32) << 16).view(np.float32)
+        amb = oracle.amax_channels(xb, axis)
+        assert np.array_equal(amb, np.abs(xw).max(axis=axis))
+        yb = xw * (s[None, :] if axis == 0 else s[:, None])
+        assert np.array_equal(oracle.quantize_channels(xb, s, axis, fmt), _nearest_code(yb, fmt))
+    # NaN propagates per channel only
+    xn = x.copy()
+    xn[5, 7] = np.nan
+    a0, a1 = oracle.amax_channels(xn, 0), oracle.amax_channels(xn, 1)
+    assert np.isnan(a0[7]) and np.isnan(a1[5]) and np.isnan(a0).sum() == 1 and np.isnan(a1).sum() == 1
+    # column-scaled GEMM = float64 matmul of the decoded codes, column j times sa_inv * sb_inv[j]
+    M, N, K = 7, 10, 48
+    A = _finite_codes(rng, E4M3, (M, K))
+    B = _finite_codes(rng, fmt, (K, N))
+    sv = np.exp2(rng.uniform(-6, 2, size=N)).astype(np.float32)
+    sa_inv = np.float32(0.37)
+    ref, sab = oracle.gemm_rows_colscale(A, E4M3, (K, 1), B, fmt, (N, 1), N, K, 0, M, sa_inv, sv)
+    da, db = oracle.decode_table(E4M3)[A], oracle.decode_table(fmt)[B]
+    alpha = np.float64(sa_inv) * sv.astype(np.float64)
+    want, want_abs = (da @ db) * alpha[None, :], (np.abs(da) @ np.abs(db)) * alpha[None, :]
+    assert np.allclose(ref, want, rtol=1e-13, atol=0) and np.allclose(sab, want_abs, rtol=1e-13, atol=0)
+    # with B stored transposed ([N, K], strides (1, K)) the same numbers come out
+    ref_t, _ = oracle.gemm_rows_colscale(A, E4M3, (K, 1), np.ascontiguousarray(B.T), fmt, (1, K), N, K, 0, M, sa_inv, sv)
+    assert np.array_equal(ref_t, ref)

@@ -3,14 +3,17 @@ allocate device memory (its control words live in a small array inside the libra
 
 Collected last on purpose: if this file fails, a run that stops at the first failure has already run
 every other test.  The check is against the existing entry point fp8_quantize_current, bit for bit
-(the tolerance every cast test uses), on two calls in a row, through the C ABI."""
+(the tolerance every cast test uses), on two calls in a row, through the C ABI; one case is also compared
+directly with the CPU oracle."""
 import ctypes
 
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2209_05433_b200 import api, synth
+from tests._util import THREADS, to_np_bits
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -57,13 +60,27 @@ def test_static_scratch_variant_matches_workspace_variant_twice_in_a_row(wide):
         assert torch.equal(o, ref) and a.item() == ra.item() and s.item() == rs.item() and si.item() == rsi.item()
 
 
+def test_static_scratch_variant_matches_the_oracle():
+    x = synth.gradients((1 << 21) + 3, 9, dtype=torch.bfloat16, device=DEV)
+    codes = torch.empty(x.numel(), dtype=torch.uint8, device=DEV)
+    a, s, si = _scalars()
+    api.fp8_quantize_current_static(x, api.E5M2, codes, a, s, si)
+    torch.cuda.synchronize()
+    xh = to_np_bits(x)
+    want_amax = oracle.amax(xh, THREADS)
+    ws, wsi = oracle.scale_from_amax(want_amax, oracle.E5M2)
+    assert a.item() == want_amax and s.item() == ws and si.item() == wsi
+    assert np.array_equal(codes.cpu().numpy(), oracle.quantize(xh, ws, oracle.E5M2, threads=THREADS))
+
+
 def test_static_scratch_variant_edge_sizes_and_limit():
     for n in (0, 1, 9, 4099):
         x = synth.activations(n, 5, dtype=torch.bfloat16, device=DEV)
         _run_pair(x, api.E4M3, api.SATURATE)
     # beyond the stated maximum: refused on the host, nothing is enqueued or dereferenced
     lib = api.load()
-    one = ctypes.c_void_p(256)
+    buf = torch.zeros(4096, dtype=torch.uint8, device=DEV)              # a real buffer: the call is refused before it is used
+    one = ctypes.c_void_p(buf.data_ptr())
     too_many = ctypes.c_size_t(api.STATIC_MAX_ELEMENTS + 1)
     status = lib.fp8_quantize_current_static(one, api.BF16, too_many, api.E4M3, api.SATURATE, one, one, one, one, None)
     assert status == 5 and lib.fp8_status_string(status) == b"unsupported size"
