@@ -152,7 +152,15 @@ __device__ __forceinline__ uint32_t quantize_item_f32(const uint4& v, float scal
 // kernels: 16-byte aligned fast path
 // ---------------------------------------------------------------------------
 
-// amax over n elements; *amax_bits must be zero before the launch.
+// One word set to zero: the start value of an amax accumulated with atomicMax by the kernel launched next.
+// It waits for everything earlier in the stream first, so the kernel behind it may read its inputs at once.
+__global__ void k_zero_word(uint32_t* p) {
+    grid_dependency_wait();
+    *p = 0u;
+}
+
+// amax over n elements.  Launched behind k_zero_word(amax_bits): the loads start while that kernel runs, only the
+// final atomicMax waits for it.
 template <int WIDE, int UNROLL>
 __global__ void __launch_bounds__(kThreads) k_amax(const void* __restrict__ x, size_t n, uint32_t* amax_bits) {
     __shared__ uint32_t red[32];
@@ -181,16 +189,20 @@ __global__ void __launch_bounds__(kThreads) k_amax(const void* __restrict__ x, s
     m = finish_abs_max<WIDE>(m);
     if (blockIdx.x == 0 && threadIdx.x < n - n_items * EPI)      // ragged tail, fewer than EPI elements
         m = max(m, canonical_nan_bits(scalar_abs_bits<WIDE>(x, n_items * EPI + threadIdx.x)));
+    grid_launch_dependents();
+    grid_dependency_wait();                                      // the accumulator has been zeroed
     block_atomic_max_bits(m, red, amax_bits);
 }
 
-// quantize n elements (+ optional amax of the input in the same pass).
+// quantize n elements (+ optional amax of the input in the same pass).  With amax the kernel is launched behind
+// k_zero_word and waits only before its atomicMax; without, it waits before its first load.
 template <int WIDE, int FMT, bool NOSAT, bool WITH_AMAX, int UNROLL>
 __global__ void __launch_bounds__(kThreads)
 k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale_dev,
            uint8_t* __restrict__ out, uint32_t* amax_bits) {
     __shared__ uint32_t red[32];
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    if (!WITH_AMAX) grid_dependency_wait();
     const float scale = *scale_dev;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
     const size_t n_items = n / EPI;
@@ -229,7 +241,11 @@ k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale
         const float xf = scalar_load<WIDE>(x, i);
         out[i] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * scale, __float_as_uint(xf));
     }
-    if (WITH_AMAX) block_atomic_max_bits(finish_abs_max<WIDE>(m), red, amax_bits);
+    grid_launch_dependents();
+    if (WITH_AMAX) {
+        grid_dependency_wait();                                  // the accumulator has been zeroed
+        block_atomic_max_bits(finish_abs_max<WIDE>(m), red, amax_bits);
+    }
 }
 
 // dequantize: 8 codes (bf16 out) or 4 codes (f32 out) per item, one 16-byte store each.
@@ -237,6 +253,7 @@ template <int FMT, int WIDE, int UNROLL>
 __global__ void __launch_bounds__(kThreads)
 k_dequantize(const uint8_t* __restrict__ c, size_t n, const float* __restrict__ scale_inv_dev, void* __restrict__ out) {
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    grid_dependency_wait();
     const float si = *scale_inv_dev;
     const size_t n_items = n / EPI;
     const size_t per_chunk = (size_t)kThreads * UNROLL;
@@ -292,6 +309,7 @@ k_dequantize(const uint8_t* __restrict__ c, size_t n, const float* __restrict__ 
         if (WIDE == kWideBF16) reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)pack_bf16(v, 0.0f);
         else                   reinterpret_cast<float*>(out)[i] = v;
     }
+    grid_launch_dependents();
 }
 
 // ---------------------------------------------------------------------------
@@ -335,6 +353,7 @@ k_dequantize_elementwise(const uint8_t* __restrict__ c, size_t n, const float* _
 
 // scale = fmax / amax with the guards of the interface; one thread.
 __global__ void k_scale_from_amax(const float* amax_dev, float fmax, float* scale_dev, float* scale_inv_dev) {
+    grid_dependency_wait();
     const float a = *amax_dev;
     float s = 1.0f;
     if (a == a && a != 0.0f && fabsf(a) != __int_as_float(0x7F800000)) {
@@ -533,6 +552,7 @@ __global__ void __launch_bounds__(kThreads)
 k_fake_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale_dev,
                 const float* __restrict__ scale_inv_dev, void* __restrict__ out) {
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    grid_dependency_wait();
     const float scale = *scale_dev, si = *scale_inv_dev;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
     const size_t n_items = n / EPI;
@@ -579,6 +599,7 @@ k_fake_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ 
         if (WIDE == kWideBF16) reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)pack_bf16(v, 0.0f);
         else                   reinterpret_cast<float*>(out)[i] = v;
     }
+    grid_launch_dependents();
 }
 
 template <int WIDE, int FMT, bool NOSAT>
@@ -597,6 +618,7 @@ k_fake_quantize_elementwise(const void* __restrict__ x, size_t n, const float* _
 // With such a scale the conversion is the paper's "programmable exponent bias" variant (Section 3.2).
 __global__ void k_scale_pow2_from_amax(const float* amax_dev, float fmax, float* scale_dev, float* scale_inv_dev) {
     float s, si;
+    grid_dependency_wait();
     scale_pair_from_amax(*amax_dev, fmax, s, si);
     uint32_t b = __float_as_uint(s);
     if ((b >> 23) != 0u) b &= 0x7F800000u;                       // normal: drop the fraction
@@ -1033,7 +1055,7 @@ static fp8_status launch_amax(const void* x, size_t n, uint32_t* bits, cudaStrea
     if (aligned16(x)) {
         auto k = k_amax<WIDE, kAmaxUnroll>;
         const int grid = persistent_grid(k, chunks_of(n, WIDE == kWideBF16 ? 8 : 4, kAmaxUnroll));
-        k<<<grid, kThreads, 0, st>>>(x, n, bits);
+        if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, bits) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_amax_elementwise<WIDE>;
         const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
@@ -1051,7 +1073,7 @@ static fp8_status launch_quantize(const void* x, size_t n, const float* scale, u
     if (aligned16(x) && (reinterpret_cast<uintptr_t>(out) & (EPI - 1)) == 0) {
         auto k = k_quantize<WIDE, FMT, NOSAT, WITH_AMAX, UNROLL>;
         const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL), kQuantPerSM);
-        k<<<grid, kThreads, 0, st>>>(x, n, scale, out, bits);
+        if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, scale, out, bits) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_quantize_elementwise<WIDE, FMT, NOSAT, WITH_AMAX>;
         const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
@@ -1075,7 +1097,7 @@ static fp8_status launch_dequantize(const uint8_t* c, size_t n, const float* si,
     if (aligned16(out) && (reinterpret_cast<uintptr_t>(c) & (EPI - 1)) == 0) {
         auto k = k_dequantize<FMT, WIDE, kDequantUnroll>;
         const int grid = persistent_grid(k, chunks_of(n, EPI, kDequantUnroll), kDequantPerSM);
-        k<<<grid, kThreads, 0, st>>>(c, n, si, out);
+        if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, c, n, si, out) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_dequantize_elementwise<FMT, WIDE>;
         const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
@@ -1085,8 +1107,10 @@ static fp8_status launch_dequantize(const uint8_t* c, size_t n, const float* si,
     return launch_status();
 }
 
+// The start value of an amax: a one-thread kernel rather than a memset node, so that the kernel behind it can be
+// scheduled, and read its inputs, while this one runs.
 static fp8_status zero_word(void* p, cudaStream_t st) {
-    if (cudaMemsetAsync(p, 0, 4, st) != cudaSuccess) return FP8_ERR_CUDA;
+    if (launch_programmatic(k_zero_word, dim3(1), dim3(1), st, reinterpret_cast<uint32_t*>(p)) != cudaSuccess) return FP8_ERR_CUDA;
     count_launches(1);
     return FP8_OK;
 }
@@ -1152,7 +1176,7 @@ static fp8_status launch_fake(const void* x, size_t n, const float* scale, const
     if (aligned16(x) && aligned16(out)) {
         auto k = k_fake_quantize<WIDE, FMT, NOSAT, UNROLL>;
         const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL), kFakePerSM);
-        k<<<grid, kThreads, 0, st>>>(x, n, scale, si, out);
+        if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, scale, si, out) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_fake_quantize_elementwise<WIDE, FMT, NOSAT>;
         const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
@@ -1307,7 +1331,9 @@ fp8_status fp8_amax(const void* x, fp8_wide t, size_t n, float* amax_dev, void* 
 fp8_status fp8_scale_from_amax(const float* amax_dev, fp8_format f, float* scale_dev, float* scale_inv_dev, void* stream) {
     if (!amax_dev || !scale_dev || !scale_inv_dev) return FP8_ERR_NULL;
     if (f != FP8_E4M3 && f != FP8_E5M2) return FP8_ERR_ENUM;
-    k_scale_from_amax<<<1, 1, 0, (cudaStream_t)stream>>>(amax_dev, f == FP8_E4M3 ? 448.0f : 57344.0f, scale_dev, scale_inv_dev);
+    if (launch_programmatic(k_scale_from_amax, dim3(1), dim3(1), (cudaStream_t)stream, amax_dev, f == FP8_E4M3 ? 448.0f : 57344.0f,
+                            scale_dev, scale_inv_dev) != cudaSuccess)
+        return FP8_ERR_CUDA;
     count_launches(1);
     return launch_status();
 }

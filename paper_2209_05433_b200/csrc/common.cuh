@@ -22,7 +22,31 @@ inline fp8_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? FP8_OK : FP8_ERR_CUDA;
 }
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the
+// stream is still draining (once every block of the predecessor has signalled or exited).  Such a kernel must
+// execute grid_dependency_wait() before it touches memory an earlier kernel may still be writing.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_programmatic(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- device side -----------------------------------------------------------
+
+// Blocks until every earlier kernel of the stream has completed and its writes are visible (no-op when the
+// kernel was launched without programmatic serialization).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream be scheduled: called once a block has issued its last load.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t ld_nc_u32(const void* p) {
     uint32_t v;
