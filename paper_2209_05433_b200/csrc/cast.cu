@@ -1,10 +1,12 @@
 // amax, scale selection, quantize (wide -> FP8) and dequantize (FP8 -> wide):
 // the memory-bound half of the FP8 hot path (Section 2 of the paper).
 //
-// The flat tensor kernels (amax, quantize, dequantize, the simulated round trip and the one-launch
-// current scaling) are persistent grid-stride loops over 16-byte items with several independent
-// 128-bit loads in flight per thread; every warp-level load and store instruction covers one
-// contiguous span.  HBM traffic is the algorithmic minimum (each input byte read once per pass, each
+// The flat tensor kernels (amax, quantize, dequantize, the simulated round trip) work on chunks of 16-byte
+// items with several independent 128-bit loads in flight per thread, one or two chunks per block, the blocks
+// handed out in order by the hardware scheduler; the one-launch current scaling is a co-resident (cooperative)
+// grid-stride loop with a grid barrier between its passes.  Every warp-level load and store instruction
+// covers one contiguous span.  Consecutive kernels of a stream overlap their launch with the predecessor's
+// tail (programmatic dependent launch).  HBM traffic is the algorithmic minimum (each input byte read once per pass, each
 // output byte written once).  The 2-D kernels (per-row / per-column scales, quantize with a transposed
 // copy) follow the same rules with shapes of their own, described at each kernel.
 #include <cuda.h>
@@ -1021,17 +1023,23 @@ k_quantize_transpose_elementwise(const void* __restrict__ x, int64_t rows, int64
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Persistent grid: enough blocks to fill every SM (at most `per_sm_cap` of them per SM), no more than there is work.
-// Kernels that mix a read and a write stream run faster with fewer resident CTAs than fit: quantize 6 per SM,
-// dequantize 3, the simulated round trip 5 (4-6 % over full residency on 2^29 bf16 elements); the read-only amax and
-// the two-pass current scaling are fastest at full residency.
-constexpr int kQuantPerSM = 6, kDequantPerSM = 3, kFakePerSM = 5, kCurrentPerSM = 64;
+// Grid of a streaming kernel: one block per `chunks_per_block` chunks, handed out by the hardware scheduler in
+// order as blocks retire.  Short-lived blocks balance the load between SMs that see different memory bandwidth: a
+// persistent grid with an equal share per block ends with a tail and measured 4 % (amax) to 12-16 % (dequantize, the
+// simulated round trip) slower on 2^28 bf16 elements.  Kernels without a reduction take one chunk per block
+// (8-16 KB of input); kernels that end in a block reduction and an atomic take 32 KB of input per block.
+static int stream_grid(size_t work_chunks, int chunks_per_block) {
+    size_t g = (work_chunks + (size_t)chunks_per_block - 1) / (size_t)chunks_per_block;
+    if (g > ((size_t)1 << 30)) g = (size_t)1 << 30;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+// Co-resident grid of the cooperative one-launch kernel: SMs x occupancy at most, no more than there is work.
 template <typename Kernel>
-static int persistent_grid(Kernel kernel, size_t work_chunks, int per_sm_cap = 64) {
+static int resident_grid(Kernel kernel, size_t work_chunks) {
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
-    // the cap pays only on long streams; a tensor of a few chunks per CTA wants every CTA it can get
-    if (per_sm > per_sm_cap && work_chunks > (size_t)4 * (size_t)sm_count() * (size_t)per_sm) per_sm = per_sm_cap;
     size_t g = (size_t)sm_count() * (size_t)per_sm;
     if (g > work_chunks) g = work_chunks;
     if (g < 1) g = 1;
@@ -1044,21 +1052,24 @@ static size_t chunks_of(size_t n, int epi, int unroll) {
     return (items + per_chunk - 1) / per_chunk;
 }
 
+// chunks per block of the kernels that end in a reduction: 32 KB of input per block in both cases
+constexpr int kAmaxChunksPerBlock = 1, kQuantAmaxChunksPerBlock = 2;
 // independent 16-byte loads in flight per thread
 constexpr int kAmaxUnroll = 8;
-constexpr int kQuantUnrollBF16 = 2;
+constexpr int kQuantUnrollBF16 = 4;
 constexpr int kQuantUnrollF32 = 8;
 constexpr int kDequantUnroll = 4;
+constexpr int kFakeUnroll = 2;
 
 template <int WIDE>
 static fp8_status launch_amax(const void* x, size_t n, uint32_t* bits, cudaStream_t st) {
     if (aligned16(x)) {
         auto k = k_amax<WIDE, kAmaxUnroll>;
-        const int grid = persistent_grid(k, chunks_of(n, WIDE == kWideBF16 ? 8 : 4, kAmaxUnroll));
+        const int grid = stream_grid(chunks_of(n, WIDE == kWideBF16 ? 8 : 4, kAmaxUnroll), kAmaxChunksPerBlock);
         if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, bits) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_amax_elementwise<WIDE>;
-        const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
+        const int grid = stream_grid((n + kThreads - 1) / kThreads, 16);
         k<<<grid, kThreads, 0, st>>>(x, n, bits);
     }
     count_launches(1);
@@ -1072,11 +1083,16 @@ static fp8_status launch_quantize(const void* x, size_t n, const float* scale, u
     // the vector path stores EPI codes per item: out must be EPI-byte aligned, x 16-byte aligned
     if (aligned16(x) && (reinterpret_cast<uintptr_t>(out) & (EPI - 1)) == 0) {
         auto k = k_quantize<WIDE, FMT, NOSAT, WITH_AMAX, UNROLL>;
-        const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL), kQuantPerSM);
+        int grid = stream_grid(chunks_of(n, EPI, UNROLL), WITH_AMAX ? kQuantAmaxChunksPerBlock : 1);
+        if (WITH_AMAX) {                                          // a small tensor still wants about seven blocks per SM
+            const size_t chunks = chunks_of(n, EPI, UNROLL), floor_blocks = (size_t)7 * (size_t)sm_count();
+            const size_t low = chunks < floor_blocks ? chunks : floor_blocks;
+            if ((size_t)grid < low) grid = (int)low;
+        }
         if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, scale, out, bits) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_quantize_elementwise<WIDE, FMT, NOSAT, WITH_AMAX>;
-        const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
+        const int grid = stream_grid((n + kThreads - 1) / kThreads, 16);
         k<<<grid, kThreads, 0, st>>>(x, n, scale, out, bits);
     }
     count_launches(1);
@@ -1096,11 +1112,11 @@ static fp8_status launch_dequantize(const uint8_t* c, size_t n, const float* si,
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
     if (aligned16(out) && (reinterpret_cast<uintptr_t>(c) & (EPI - 1)) == 0) {
         auto k = k_dequantize<FMT, WIDE, kDequantUnroll>;
-        const int grid = persistent_grid(k, chunks_of(n, EPI, kDequantUnroll), kDequantPerSM);
+        const int grid = stream_grid(chunks_of(n, EPI, kDequantUnroll), 1);
         if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, c, n, si, out) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_dequantize_elementwise<FMT, WIDE>;
-        const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
+        const int grid = stream_grid((n + kThreads - 1) / kThreads, 16);
         k<<<grid, kThreads, 0, st>>>(c, n, si, out);
     }
     count_launches(1);
@@ -1123,7 +1139,7 @@ static fp8_status launch_current(const void* x, size_t n, float fmax, uint8_t* o
     auto k = k_quantize_current<WIDE, FMT, NOSAT, UNROLL>;
     size_t chunks = chunks_of(n, EPI, UNROLL);
     if (chunks < 1) chunks = 1;
-    const int grid = persistent_grid(k, chunks, kCurrentPerSM);   // co-resident by construction: SMs x occupancy at most
+    const int grid = resident_grid(k, chunks);
     unsigned int arrivals = (unsigned int)grid;
     long long wait_limit = kGridWaitLimitCycles;
     void* args[] = {(void*)&x, (void*)&n, (void*)&fmax, (void*)&out, (void*)&amax, (void*)&scale, (void*)&scale_inv, (void*)&ws,
@@ -1172,14 +1188,14 @@ fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_form
 template <int WIDE, int FMT, bool NOSAT>
 static fp8_status launch_fake(const void* x, size_t n, const float* scale, const float* si, void* out, cudaStream_t st) {
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
-    constexpr int UNROLL = 2;
+    constexpr int UNROLL = kFakeUnroll;
     if (aligned16(x) && aligned16(out)) {
         auto k = k_fake_quantize<WIDE, FMT, NOSAT, UNROLL>;
-        const int grid = persistent_grid(k, chunks_of(n, EPI, UNROLL), kFakePerSM);
+        const int grid = stream_grid(chunks_of(n, EPI, UNROLL), 1);
         if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, scale, si, out) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_fake_quantize_elementwise<WIDE, FMT, NOSAT>;
-        const int grid = persistent_grid(k, (n + kThreads - 1) / kThreads);
+        const int grid = stream_grid((n + kThreads - 1) / kThreads, 16);
         k<<<grid, kThreads, 0, st>>>(x, n, scale, si, out);
     }
     count_launches(1);

@@ -115,6 +115,9 @@ def _linear_layer(seed, T, I, O, w_sigma, passes, n_random):
         Y = torch.empty(T, O, dtype=torch.bfloat16, device=DEV)
         api.fp8_gemm(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, six, siw, amax)
         _check_gemm(Y, amax, Xh, E4, (I, 1), Wh, E4, (O, 1), I, wsix, wsiw, rng, "fprop K=%d" % I, n_random)
+        # the same product with split accumulation (partial sums every 2048 of K added in registers)
+        api.fp8_gemm(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, six, siw, amax, acc=api.ACC_SPLIT)
+        _check_gemm(Y, amax, Xh, E4, (I, 1), Wh, E4, (O, 1), I, wsix, wsiw, rng, "fprop K=%d split accumulation" % I, n_random // 8, 4)
         del Y
     if "dgrad" in passes or "wgrad" in passes:
         dY = synth.gradients(T * O, seed, device=DEV).view(T, O)
@@ -134,6 +137,8 @@ def _linear_layer(seed, T, I, O, w_sigma, passes, n_random):
             dW = torch.empty(I, O, dtype=torch.bfloat16, device=DEV)
             api.fp8_gemm(Xq, api.E4M3, api.MAJOR_MN, Gq, api.E5M2, api.MAJOR_MN, dW, six, sig, amax)
             _check_gemm(dW, amax, Xh, E4, (1, I), Gh, E5, (O, 1), T, wsix, wsig, rng, "wgrad K=%d" % T, n_random)
+            api.fp8_gemm(Xq, api.E4M3, api.MAJOR_MN, Gq, api.E5M2, api.MAJOR_MN, dW, six, sig, amax, acc=api.ACC_SPLIT)
+            _check_gemm(dW, amax, Xh, E4, (1, I), Gh, E5, (O, 1), T, wsix, wsig, rng, "wgrad K=%d split accumulation" % T, n_random // 8, 4)
             del dW
     torch.cuda.empty_cache()
 
