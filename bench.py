@@ -449,9 +449,10 @@ def bench_next_rows(torch, api, synth, device, pk, iters=5):
 _oracle_inputs = {}
 
 
-def oracle_step(layer: str, sample_tokens: int, threads: int, sample_out: int | None = None):
+def oracle_step(layer: str, sample_tokens: int, threads: int, sample_out: int | None = None, inputs=None):
     """The same step on a bounded sample of the layer: `sample_tokens` tokens and `sample_out` output features
-    (W is [d_in, sample_out], same recipe), run by the CPU oracle as it stands.
+    (W is [d_in, sample_out], same recipe), run by the CPU oracle as it stands.  `inputs` = (X, W, dY) as bf16 bit
+    patterns of exactly that sample (the GPU arm passes slices of its own tensors); otherwise they are generated here.
     Returns (seconds, gemm flops of the sample)."""
     import numpy as np
     import torch
@@ -466,6 +467,9 @@ def oracle_step(layer: str, sample_tokens: int, threads: int, sample_out: int | 
         return t.view(torch.int16).numpy().view(np.uint16)
 
     key = (layer, T, O)
+    if inputs is not None:
+        _oracle_inputs.clear()
+        _oracle_inputs[key] = inputs
     if key not in _oracle_inputs:                                  # synthetic inputs are made once, outside the timed part
         _oracle_inputs.clear()
         _oracle_inputs[key] = (bits(synth.activations(T * I, L["seed"], dtype=torch.bfloat16)),
@@ -478,13 +482,19 @@ def oracle_step(layer: str, sample_tokens: int, threads: int, sample_out: int | 
         s, si = oracle.scale_from_amax(oracle.amax(t, threads), fmt)
         q[name], sinv[name] = oracle.quantize(t, s, fmt, threads=threads), si
     oracle.dequantize(q["x"], sinv["x"], oracle.E4M3, "bf16", threads=threads)
+    def product(A, fa, a_str, B, fb, b_str, rows, cols, k, sa, sb):
+        """every output element of a rows x cols product through the oracle's per-element routine; the element list
+        (not the few rows of the sample) is what is split over the host cores"""
+        ii, jj = np.repeat(np.arange(rows, dtype=np.int64), cols), np.tile(np.arange(cols, dtype=np.int64), rows)
+        return oracle.gemm_samples(A, fa, a_str, B, fb, b_str, k, ii, jj, sa, sb, threads=threads)[0]
+
     results = []
     if "fprop" in L["passes"]:
-        results.append(oracle.gemm_rows(q["x"], oracle.E4M3, (I, 1), q["w"], oracle.E4M3, (O, 1), O, I, 0, T, sinv["x"], sinv["w"], threads)[0])
+        results.append(product(q["x"], oracle.E4M3, (I, 1), q["w"], oracle.E4M3, (O, 1), T, O, I, sinv["x"], sinv["w"]))
     if "dgrad" in L["passes"]:
-        results.append(oracle.gemm_rows(q["g"], oracle.E5M2, (O, 1), q["w"], oracle.E4M3, (1, O), I, O, 0, T, sinv["g"], sinv["w"], threads)[0])
+        results.append(product(q["g"], oracle.E5M2, (O, 1), q["w"], oracle.E4M3, (1, O), T, I, O, sinv["g"], sinv["w"]))
     if "wgrad" in L["passes"]:
-        results.append(oracle.gemm_rows(q["x"], oracle.E4M3, (1, I), q["g"], oracle.E5M2, (O, 1), O, T, 0, I, sinv["x"], sinv["g"], threads)[0])
+        results.append(product(q["x"], oracle.E4M3, (1, I), q["g"], oracle.E5M2, (O, 1), I, O, T, sinv["x"], sinv["g"]))
     for r in results:
         oracle.round_bf16_from_f64(r)
     dt = time.perf_counter() - t0
@@ -738,9 +748,11 @@ def run_ours(args, world, rank, local):
         # the memory-bound half: amax + quantize (+ dequantize) of the step against HBM
         c_sus, c_burst = sus["cast_total_gbs"], burst["cast_total_gbs"]
         roofline_cast = {
-            "bound": "hbm", "kernel": "casts of the step: k_quantize_current (X, W, dY) + k_dequantize", "achieved": round(c_sus, 1),
+            "bound": "hbm", "kernel": "casts of the step: current scaling of X (one cooperative k_quantize_current), of W and dY (k_amax + k_scale_from_amax + k_quantize each, tensors of 256 MB and more) + k_dequantize", "achieved": round(c_sus, 1),
             "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": round(c_sus / pk["hbm_gbs"], 4),
-            "traffic": traffic.get("k_quantize_current.W." + layer),
+            "traffic": traffic.get("cast_W." + layer),
+            "traffic_note": "DRAM bytes of one current-scaling call on W (the amax and the quantize kernel together) from the ncu capture "
+                            "summarised under profiles/; algorithmic %.3e" % (5.0 * step.I * step.O),
             "peak_source": pk["source"] + " copy bandwidth", "regime": "sustained loop (same as roofline)",
             "per_call_gbs": sus["cast_gbs"], "burst": {"achieved": round(c_burst, 1), "frac": round(c_burst / pk["hbm_gbs"], 4), "per_call_gbs": burst["cast_gbs"]},
             "frac_of_nominal_8000": round(c_sus / NOMINAL_HBM_GBS, 4),
@@ -752,6 +764,10 @@ def run_ours(args, world, rank, local):
                      "kernels": sus["kernels"]}
         per_config = cast_sizes = next_rows = cpu = None
         if world == 1 and not args.quick:
+            threads = os.cpu_count() or 1
+            cpu_tokens = 4 if threads >= 12 else 2                 # about 20 s of CPU work on 16 cores
+            to_bits = lambda t: t.contiguous().cpu().view(torch.int16).numpy().view("uint16").reshape(-1)
+            cpu_inputs = (to_bits(step.X[:cpu_tokens]), to_bits(step.W), to_bits(step.dY[:cpu_tokens]))
             del step
             torch.cuda.empty_cache()
             cast_sizes = bench_cast_sizes(torch, api, synth, device, pk)
@@ -766,9 +782,7 @@ def run_ours(args, world, rank, local):
             del small
             torch.cuda.empty_cache()
             next_rows = bench_next_rows(torch, api, synth, device, pk)
-            threads = os.cpu_count() or 1
-            cpu_tokens = 2 if threads >= 12 else 1                 # about 20 s of CPU work on 16 cores
-            dt, flops = oracle_step(layer, cpu_tokens, threads)
+            dt, flops = oracle_step(layer, cpu_tokens, threads, inputs=cpu_inputs)
             cpu = {"value": flops / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": round(dt, 2),
                    "sample": "the same step with %d of the %d tokens (weights at full size), CPU oracle as it stands" % (cpu_tokens, LAYERS[layer]["tokens"])}
         L = LAYERS[layer]

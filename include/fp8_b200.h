@@ -93,13 +93,16 @@ fp8_status fp8_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_o
                         const float* scale_dev, uint8_t* out, float* amax_dev, void* stream);
 
 /*
- * fp8_quantize_current — Section 2, the whole "current scaling" conversion of one tensor in ONE launch:
+ * fp8_quantize_current — Section 2, the whole "current scaling" conversion of one tensor in ONE call:
  * the scale is chosen from the tensor's own maximum magnitude, then the tensor is converted with it.
  * Results are identical, bit for bit, to fp8_amax + fp8_scale_from_amax + fp8_quantize:
  *   *amax_dev = amax(x); *scale_dev = fmax/amax (same guards); *scale_inv_dev = 1/scale;
  *   out_i = encode_f( binary32(x_i) * scale ).
- * The kernel is launched cooperatively (all of its blocks resident at once) and crosses one grid-wide
- * barrier between the two passes; the second pass re-reads the tail of x from L2.
+ * Tensors below 256 MB take ONE kernel, launched cooperatively (all of its blocks resident at once), which
+ * crosses one grid-wide barrier between the two passes; the second pass re-reads the tail of x from L2.
+ * Larger tensors (and pointers without 16-byte alignment) take the three streaming kernels back to back on the
+ * stream, the conversion walking the tensor from its end, where the amax pass has just been: on long streams
+ * that is the faster form, and the workspace is then not touched.
  *   workspace  device, fp8_quantize_current_workspace_bytes() bytes, 16-byte aligned, owned by the
  *              caller.  It must hold zeros before the first call; every call leaves it zeroed again,
  *              so one buffer serves any number of calls on one stream.  Calls that may overlap on the
@@ -211,6 +214,10 @@ fp8_status fp8_scale_pow2_from_amax(const float* amax_dev, fp8_format f,
  *   magnitude inside the bound at every K of the workloads; a caller whose products share one sign over a long K
  *   (K > 2048) should ask for SPLIT.
  * Every GEMM entry point that takes this descriptor honours `acc`; other values give FP8_ERR_ENUM.
+ * Reproducibility: a call is bit-reproducible for a given problem (shapes, layouts, data) on a given device.  The
+ * order in which the K-blocks of an output tile are accumulated (from the start or from the end of K) depends on
+ * the tile's place in the kernel's schedule, so two equal dot products in different tiles may differ in the last
+ * bits, within the stated tolerance.
  */
 typedef struct {
     int64_t M, N, K;

@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(kThreads) k_amax(const void* __restrict__ x, s
 template <int WIDE, int FMT, bool NOSAT, bool WITH_AMAX, int UNROLL>
 __global__ void __launch_bounds__(kThreads)
 k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale_dev,
-           uint8_t* __restrict__ out, uint32_t* amax_bits) {
+           uint8_t* __restrict__ out, uint32_t* amax_bits, int reverse) {
     __shared__ uint32_t red[32];
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
     if (!WITH_AMAX) grid_dependency_wait();
@@ -218,8 +218,9 @@ k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale
         else                   st_out(reinterpret_cast<uint32_t*>(out) + i, quantize_item_f32<FMT, NOSAT>(v, scale));
     };
 
+    // `reverse`: the first blocks take the last chunks (the part of x a preceding amax pass read last is still in L2)
     for (size_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
-        const size_t base = chunk * per_chunk + threadIdx.x;
+        const size_t base = (reverse ? n_chunks - 1 - chunk : chunk) * per_chunk + threadIdx.x;
         if (base + (size_t)(UNROLL - 1) * kThreads < n_items) {
             uint4 v[UNROLL];
 #pragma unroll
@@ -385,6 +386,10 @@ constexpr long long kGridWaitLimitCycles = 4000000000ll;       // about 2 s of S
 // the first pass are asked to stay in L2 (the second pass starts there), the rest to leave first.  Smaller tensors
 // are left to the default replacement: they mostly fit.
 constexpr size_t kCurrentKeepMB = 96, kCurrentKeepFromMB = 160;
+// From this input size on, fp8_quantize_current runs the three streaming kernels instead of the one cooperative
+// launch: their scheduler-balanced blocks beat the co-resident grid on long streams (2^28 bf16 elements: +2 %,
+// 2^30: +8 %), where a few launch gaps do not show; below it the two are within noise of each other.
+constexpr size_t kCurrentChainFromBytes = (size_t)256 << 20;
 __device__ __forceinline__ uint64_t l2_policy_evict_last() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
@@ -1077,7 +1082,8 @@ static fp8_status launch_amax(const void* x, size_t n, uint32_t* bits, cudaStrea
 }
 
 template <int WIDE, int FMT, bool NOSAT, bool WITH_AMAX>
-static fp8_status launch_quantize(const void* x, size_t n, const float* scale, uint8_t* out, uint32_t* bits, cudaStream_t st) {
+static fp8_status launch_quantize(const void* x, size_t n, const float* scale, uint8_t* out, uint32_t* bits, cudaStream_t st,
+                                  int reverse = 0) {
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
     constexpr int UNROLL = WIDE == kWideBF16 ? kQuantUnrollBF16 : kQuantUnrollF32;
     // the vector path stores EPI codes per item: out must be EPI-byte aligned, x 16-byte aligned
@@ -1089,7 +1095,7 @@ static fp8_status launch_quantize(const void* x, size_t n, const float* scale, u
             const size_t low = chunks < floor_blocks ? chunks : floor_blocks;
             if ((size_t)grid < low) grid = (int)low;
         }
-        if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, scale, out, bits) != cudaSuccess) return FP8_ERR_CUDA;
+        if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, scale, out, bits, reverse) != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_quantize_elementwise<WIDE, FMT, NOSAT, WITH_AMAX>;
         const int grid = stream_grid((n + kThreads - 1) / kThreads, 16);
@@ -1100,11 +1106,27 @@ static fp8_status launch_quantize(const void* x, size_t n, const float* scale, u
 }
 
 template <int WIDE, int FMT>
-static fp8_status dispatch_quantize(const void* x, size_t n, bool nosat, const float* scale, uint8_t* out, uint32_t* bits, cudaStream_t st) {
-    if (nosat) return bits ? launch_quantize<WIDE, FMT, true, true>(x, n, scale, out, bits, st)
-                           : launch_quantize<WIDE, FMT, true, false>(x, n, scale, out, bits, st);
-    return bits ? launch_quantize<WIDE, FMT, false, true>(x, n, scale, out, bits, st)
-                : launch_quantize<WIDE, FMT, false, false>(x, n, scale, out, bits, st);
+static fp8_status dispatch_quantize(const void* x, size_t n, bool nosat, const float* scale, uint8_t* out, uint32_t* bits, cudaStream_t st,
+                                    int reverse = 0) {
+    if (nosat) return bits ? launch_quantize<WIDE, FMT, true, true>(x, n, scale, out, bits, st, reverse)
+                           : launch_quantize<WIDE, FMT, true, false>(x, n, scale, out, bits, st, reverse);
+    return bits ? launch_quantize<WIDE, FMT, false, true>(x, n, scale, out, bits, st, reverse)
+                : launch_quantize<WIDE, FMT, false, false>(x, n, scale, out, bits, st, reverse);
+}
+
+// amax -> scale -> quantize of one tensor as the three streaming kernels back to back (identical results to the
+// one-launch kernel); the quantize pass walks the tensor from its end, where the amax pass has just been.
+static fp8_status quantize_current_chain(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o, uint8_t* out,
+                                         float* amax, float* scale, float* scale_inv, cudaStream_t st) {
+    fp8_status s = fp8_amax(x, t, n, amax, st);
+    if (s == FP8_OK) s = fp8_scale_from_amax(amax, f, scale, scale_inv, st);
+    if (s != FP8_OK || n == 0) return s;
+    const bool nosat = o == FP8_NOSAT;
+    if (t == FP8_F32)
+        return f == FP8_E4M3 ? dispatch_quantize<kWideF32, kE4M3>(x, n, nosat, scale, out, nullptr, st, 1)
+                             : dispatch_quantize<kWideF32, kE5M2>(x, n, nosat, scale, out, nullptr, st, 1);
+    return f == FP8_E4M3 ? dispatch_quantize<kWideBF16, kE4M3>(x, n, nosat, scale, out, nullptr, st, 1)
+                         : dispatch_quantize<kWideBF16, kE5M2>(x, n, nosat, scale, out, nullptr, st, 1);
 }
 
 template <int FMT, int WIDE>
@@ -1157,12 +1179,9 @@ static fp8_status launch_current(const void* x, size_t n, float fmax, uint8_t* o
 fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o, uint8_t* out,
                                    float* amax, float* scale, float* scale_inv, unsigned int* ws, cudaStream_t st) {
     const int epi = t == FP8_BF16 ? 8 : 4;
-    if (n == 0 || !aligned16(x) || (reinterpret_cast<uintptr_t>(out) & (epi - 1)) != 0) {
-        fp8_status s = fp8_amax(x, t, n, amax, st);
-        if (s == FP8_OK) s = fp8_scale_from_amax(amax, f, scale, scale_inv, st);
-        if (s == FP8_OK) s = fp8_quantize(x, t, n, f, o, scale, out, nullptr, st);
-        return s;
-    }
+    const size_t bytes = n * (t == FP8_BF16 ? 2 : 4);
+    if (n == 0 || !aligned16(x) || (reinterpret_cast<uintptr_t>(out) & (epi - 1)) != 0 || bytes >= kCurrentChainFromBytes)
+        return quantize_current_chain(x, t, n, f, o, out, amax, scale, scale_inv, st);
     const float fmax = f == FP8_E4M3 ? 448.0f : 57344.0f;
     const bool nosat = o == FP8_NOSAT;
     fp8_status s;
@@ -1177,11 +1196,8 @@ fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_form
         else               s = nosat ? launch_current<kWideBF16, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
                                      : launch_current<kWideBF16, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
     }
-    if (s == FP8_ERR_UNSUPPORTED) {                                // cooperative launch refused: same results, three launches
-        s = fp8_amax(x, t, n, amax, st);
-        if (s == FP8_OK) s = fp8_scale_from_amax(amax, f, scale, scale_inv, st);
-        if (s == FP8_OK) s = fp8_quantize(x, t, n, f, o, scale, out, nullptr, st);
-    }
+    if (s == FP8_ERR_UNSUPPORTED)                                  // cooperative launch refused: same results, three kernels
+        s = quantize_current_chain(x, t, n, f, o, out, amax, scale, scale_inv, st);
     return s;
 }
 

@@ -47,6 +47,7 @@ constexpr int BK = 128;             // K-block in elements = bytes = one 128B sw
 constexpr int UMMA_K = 32;          // K of one tcgen05.mma for 8-bit operands
 constexpr int MAX_STAGES = 6;
 constexpr int ACC_STAGES = 2;       // 2 x 256 columns = all 512 TMEM columns
+constexpr int GROUP_M = 16;         // tile raster: GROUP_M row-tiles share each sweep over N
 // Epilogue width: 4 warps with two staging buffers each (long K: the epilogue has slack, fewer resident warps
 // leave the MMA-issuing thread undisturbed) or 8 warps (short K: the kernel is bound by its output stream; two
 // warps per TMEM lane quarter split the tile's columns and each warp has three buffers, two ring stages' worth).
@@ -68,7 +69,6 @@ constexpr uint32_t SMEM_EPI = 8 * EPI_BUF_BYTES;                    // staging b
 constexpr uint32_t SMEM_BARRIERS = 256;
 constexpr uint32_t SMEM_BYTES = SMEM_TILES + SMEM_EPI + SMEM_BARRIERS + 1024;   // + slack to align the ring to 1024 B
 constexpr uint32_t TMEM_COLS = 512;
-constexpr int GROUP_M = 16;         // tile raster: GROUP_M row-tiles share each sweep over N
 
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clocks per wait
 
@@ -377,19 +377,24 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         const uint64_t keep = policy_evict_last();
+        int tile_no = 0;
         for (int t = worker; t < num_tiles && ok; t += num_workers) {
             int tm, tn;
             const int bi = t / tiles_per_batch;                                 // batch member
             tile_coords(t - bi * tiles_per_batch, p.tiles_m, p.tiles_n, tm, tn);
             const int m0 = tm * G::TILE_M + (int)cta_rank * BM;                 // this CTA's 128 rows of A
             const int n0 = tn * BN + (int)cta_rank * (BN / CG);                 // this CTA's rows of B
+            // Every second tile of a worker walks K from its end: the workers of a wave finish a tile together at one end
+            // of their operand panels and start the next tile there, where L2 still holds what they share (measured
+            // 10-28 % fewer DRAM reads on four of the five workload GEMMs, +1.5-2.8 % sustained throughput on three).
+            const bool backwards = (tile_no++ & 1) != 0;
             for (int kb = 0; kb < k_pad; ++kb) {
                 ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, WAIT_EMPTY);
                 if (!ok) break;
                 if (lane == 0) {
                     const uint32_t sa = ring + stage * STAGE_BYTES;
                     const uint32_t sb = sa + A_BYTES;
-                    const int k0 = kb * BK;
+                    const int k0 = (backwards && kb < k_blocks ? k_blocks - 1 - kb : kb) * BK;
                     const uint32_t pair_bar = smem_u32(&bars->full[stage / FG]);          // one barrier per FG stages
                     if (CG == 2) {
                         const uint32_t full = map_to_cta(pair_bar, 0);                    // the leader's barrier

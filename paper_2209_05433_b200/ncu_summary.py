@@ -7,8 +7,9 @@ Two inputs are understood:
   * the raw page of a report,
         ncu -i report.ncu-rep --page raw --csv > raw.csv
     (one row per launch, one column per metric): prints the chosen counters per launch and, with
-    --traffic NAME, rewrites the line NAME of profiles/dram_traffic.txt with the mean DRAM bytes
-    (read + write) per launch, the figure bench.py reports as roofline.traffic.
+    --traffic NAME, rewrites the line NAME of profiles/dram_traffic.txt with the DRAM bytes (read + write)
+    per call (mean per launch of each captured kernel, summed over the kernels), the figure bench.py
+    reports as roofline.traffic.
 
     python -m paper_2209_05433_b200.ncu_summary launches.csv
     python -m paper_2209_05433_b200.ncu_summary raw.csv --kernel k_gemm_fp8 --traffic k_gemm_fp8.fprop.hidden12288
@@ -73,7 +74,7 @@ def raw_page(rows, kernel: str | None, traffic_key: str | None) -> str:
     head, units = rows[0], rows[1]
     k_name = head.index("Kernel Name")
     cols = [(c, head.index(c)) for c in COUNTERS if c in head]
-    out, traffic = [], []
+    out, traffic, names = [], [], []
     for r in rows[2:]:
         if kernel and kernel not in r[k_name]:
             continue
@@ -86,14 +87,19 @@ def raw_page(rows, kernel: str | None, traffic_key: str | None) -> str:
             rd = vals["dram__bytes_read.sum"][0] * SCALE.get(vals["dram__bytes_read.sum"][1], 1.0)
             wr = vals["dram__bytes_write.sum"][0] * SCALE.get(vals["dram__bytes_write.sum"][1], 1.0)
             traffic.append(rd + wr)
+            names.append(_short(r[k_name]))
             out.append("  %-82s %14.4e byte" % ("dram bytes read + written", rd + wr))
     if traffic_key and traffic:
-        mean = sum(traffic) / len(traffic)
+        # bytes per CALL: the mean over the launches of each kernel, summed over the kernels captured
+        per_kernel = {}
+        for name, t in zip(names, traffic):
+            per_kernel.setdefault(name, []).append(t)
+        mean = sum(sum(v) / len(v) for v in per_kernel.values())
         lines = []
         if os.path.exists(TRAFFIC_FILE):
             with open(TRAFFIC_FILE) as f:
                 lines = [l.rstrip("\n") for l in f if l.split()[:1] != [traffic_key]]
-        lines.append("%s %.6e   # mean of %d captured launches" % (traffic_key, mean, len(traffic)))
+        lines.append("%s %.6e   # %d captured launches of %s" % (traffic_key, mean, len(traffic), " + ".join(sorted(per_kernel))))
         with open(TRAFFIC_FILE, "w") as f:
             f.write("\n".join(lines) + "\n")
         out.append("wrote %s = %.6e to %s" % (traffic_key, mean, os.path.relpath(TRAFFIC_FILE, ROOT)))
