@@ -231,24 +231,16 @@ def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: in
     ``mb == MAJOR_MN``.  Row pitches are taken from the tensors' strides.
     ``acc`` selects one accumulator over all of K (ACC_FAST) or partial sums every 2048 of K added in
     registers (ACC_SPLIT: tolerance met on same-sign data at any K)."""
-    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
-        raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D tensor")
-    for t, name in ((A, "A"), (B, "B"), (D, "D")):
-        if not t.is_cuda or t.stride(1) != 1:
-            raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
-    M, K = (A.shape[0], A.shape[1]) if ma == MAJOR_K else (A.shape[1], A.shape[0])
-    Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
-    if K != Kb or tuple(D.shape) != (M, N):
-        raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
-    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D), acc)
+    d = _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc)
     _check(load().fp8_gemm(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
                            _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
                            None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()), "fp8_gemm")
 
 
-def _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc):
-    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
-        raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D tensor")
+def _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc, codes_out=False):
+    """descriptor of a 2-D product from the tensors' shapes and strides; D is a wide tensor, or uint8 codes"""
+    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2 or (codes_out and D.dtype != torch.uint8):
+        raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D %s tensor" % ("uint8" if codes_out else "float32 or bfloat16"))
     for t, name in ((A, "A"), (B, "B"), (D, "D")):
         if not t.is_cuda or t.stride(1) != 1:
             raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
@@ -256,7 +248,7 @@ def _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc):
     Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
     if K != Kb or tuple(D.shape) != (M, N):
         raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
-    return GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D), acc)
+    return GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), BF16 if codes_out else _wide_of(D), acc)
 
 
 def fp8_gemm_splitk_workspace(M: int, N: int, K: int) -> tuple[int, int]:
@@ -285,16 +277,7 @@ def fp8_gemm_fp8out(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int,
                     amax_out: torch.Tensor | None = None, overflow: int = SATURATE, acc: int = ACC_FAST) -> None:
     """D[M,N] (uint8 codes of format fd) = encode((A . B) * scale_inv_a * scale_inv_b * scale_d); amax_out
     receives the amax of the result before the output scale and conversion.  Layout rules as fp8_gemm."""
-    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or D.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
-        raise TypeError("A, B and D must be 2-D uint8 tensors")
-    for t, name in ((A, "A"), (B, "B"), (D, "D")):
-        if not t.is_cuda or t.stride(1) != 1:
-            raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
-    M, K = (A.shape[0], A.shape[1]) if ma == MAJOR_K else (A.shape[1], A.shape[0])
-    Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
-    if K != Kb or tuple(D.shape) != (M, N):
-        raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
-    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), BF16, acc)
+    d = _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc, codes_out=True)
     _check(load().fp8_gemm_fp8out(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(), fd, overflow,
                                   _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
                                   _scalar(scale_d, "scale_d"), None if amax_out is None else _scalar(amax_out, "amax_out"),
@@ -358,18 +341,9 @@ def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, 
                             scale_inv_a: torch.Tensor, scale_inv_b_vec: torch.Tensor, amax_out: torch.Tensor | None = None,
                             acc: int = ACC_FAST) -> None:
     """fp8_gemm with one inverse scale per column of B (per output channel)."""
-    if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 2 or B.dim() != 2 or D.dim() != 2:
-        raise TypeError("A and B must be 2-D uint8 tensors and D a 2-D tensor")
-    for t, name in ((A, "A"), (B, "B"), (D, "D")):
-        if not t.is_cuda or t.stride(1) != 1:
-            raise ValueError("%s must be a CUDA tensor with unit inner stride" % name)
-    M, K = (A.shape[0], A.shape[1]) if ma == MAJOR_K else (A.shape[1], A.shape[0])
-    Kb, N = (B.shape[1], B.shape[0]) if mb == MAJOR_K else (B.shape[0], B.shape[1])
-    if K != Kb or tuple(D.shape) != (M, N):
-        raise ValueError("shape mismatch: A gives M=%d K=%d, B gives K=%d N=%d, D is %s" % (M, K, Kb, N, tuple(D.shape)))
-    d = GemmDesc(M, N, K, fa, fb, ma, mb, A.stride(0), B.stride(0), D.stride(0), _wide_of(D), acc)
+    d = _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc)
     _check(load().fp8_gemm_channel_scales(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
-                                          _scalar(scale_inv_a, "scale_inv_a"), _vec(scale_inv_b_vec, N, "scale_inv_b_vec"),
+                                          _scalar(scale_inv_a, "scale_inv_a"), _vec(scale_inv_b_vec, d.N, "scale_inv_b_vec"),
                                           None if amax_out is None else _scalar(amax_out, "amax_out"), _stream()),
            "fp8_gemm_channel_scales")
 
