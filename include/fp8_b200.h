@@ -366,6 +366,18 @@ fp8_status fp8_async_status(uint32_t* detail);
 typedef enum { FP8_WAIT_MBARRIER = 0, FP8_WAIT_GRID_BARRIER = 1 } fp8_wait_kind;
 fp8_status fp8_self_test_expire_wait(int which, uint64_t limit_cycles, void* stream);
 
+/*
+ * fp8_sm_clock_probe — the paper has no counterpart; a measurement aid.  Launches a one-warp kernel that reads the SM
+ * cycle counter and the device's nanosecond timer, waits `duration_us` microseconds (1 .. 100000, else
+ * FP8_ERR_UNSUPPORTED; the wait is bounded by an iteration count as well) and reads both again.
+ *   out_dev  device, two 64-bit words, OVERWRITTEN: [0] = SM clocks elapsed, [1] = nanoseconds elapsed;
+ *            clocks * 1000 / nanoseconds = SM clock in MHz during the window.
+ * Enqueued on a second stream it runs beside other kernels (it needs one warp and no shared memory), which is how the
+ * benchmark reads the clock the tensor cores actually ran at under the power cap: the management interface samples
+ * too coarsely for that.
+ */
+fp8_status fp8_sm_clock_probe(uint64_t* out_dev, uint32_t duration_us, void* stream);
+
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* fp8_status_string(fp8_status s);
 

@@ -25,7 +25,7 @@ EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_curr
            "fp8_scale_pow2_from_amax", "fp8_gemm", "fp8_gemm_fp8out", "fp8_amax_channels", "fp8_scales_from_amax",
            "fp8_quantize_channels", "fp8_quantize_transpose", "fp8_gemm_channel_scales", "fp8_gemm_batched",
            "fp8_gemm_splitk", "fp8_gemm_splitk_workspace",
-           "fp8_async_status", "fp8_self_test_expire_wait", "fp8_status_string", "fp8_launch_count"]
+           "fp8_async_status", "fp8_self_test_expire_wait", "fp8_sm_clock_probe", "fp8_status_string", "fp8_launch_count"]
 
 
 class Fp8Error(RuntimeError):
@@ -104,6 +104,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.fp8_async_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
     lib.fp8_self_test_expire_wait.restype = i32
     lib.fp8_self_test_expire_wait.argtypes = [i32, ctypes.c_uint64, vp]
+    lib.fp8_sm_clock_probe.restype = i32
+    lib.fp8_sm_clock_probe.argtypes = [vp, ctypes.c_uint32, vp]
     lib.fp8_status_string.restype = ctypes.c_char_p
     lib.fp8_status_string.argtypes = [i32]
     lib.fp8_launch_count.restype = ctypes.c_uint64
@@ -389,6 +391,14 @@ def fp8_async_status() -> tuple[int, int]:
 def fp8_self_test_expire_wait(which: int, limit_cycles: int = 2_000_000) -> None:
     """Makes one bounded device-side wait run out on purpose (about a millisecond by default); see the header."""
     _check(load().fp8_self_test_expire_wait(which, limit_cycles, _stream()), "fp8_self_test_expire_wait")
+
+
+def fp8_sm_clock_probe(out: torch.Tensor, duration_us: int = 200) -> None:
+    """Enqueues the one-warp clock probe on the current stream; `out` is a 2-element int64 CUDA tensor that receives
+    (SM clocks, nanoseconds) of a window of `duration_us` microseconds."""
+    if out.dtype != torch.int64 or out.numel() != 2:
+        raise TypeError("out must be a 2-element int64 CUDA tensor")
+    _check(load().fp8_sm_clock_probe(_dev(out, "out"), duration_us, _stream()), "fp8_sm_clock_probe")
 
 
 def fp8_launch_count() -> int:

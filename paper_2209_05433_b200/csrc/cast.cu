@@ -354,6 +354,20 @@ k_dequantize_elementwise(const uint8_t* __restrict__ c, size_t n, const float* _
     }
 }
 
+// SM clock probe: one thread reads the SM cycle counter and the nanosecond timer, waits `duration_ns` (bounded
+// by an iteration count as well), reads both again.  out[0] = SM clocks, out[1] = nanoseconds.
+__global__ void k_sm_clock_probe(unsigned long long* out, unsigned long long duration_ns) {
+    if (threadIdx.x != 0) return;
+    unsigned long long t0, t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    const long long c0 = clock64();
+    t = t0;
+    for (unsigned int i = 0; i < 50000000u && t - t0 < duration_ns; ++i) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    const long long c1 = clock64();
+    out[0] = (unsigned long long)(c1 - c0);
+    out[1] = t - t0;
+}
+
 // scale = fmax / amax with the guards of the interface; one thread.
 __global__ void k_scale_from_amax(const float* amax_dev, float fmax, float* scale_dev, float* scale_inv_dev) {
     grid_dependency_wait();
@@ -1563,6 +1577,14 @@ fp8_status fp8_dequantize(const uint8_t* c, size_t n, fp8_format f, const float*
                              : launch_dequantize<kE5M2, kWideF32>(c, n, scale_inv_dev, out, st);
     return f == FP8_E4M3 ? launch_dequantize<kE4M3, kWideBF16>(c, n, scale_inv_dev, out, st)
                          : launch_dequantize<kE5M2, kWideBF16>(c, n, scale_inv_dev, out, st);
+}
+
+fp8_status fp8_sm_clock_probe(uint64_t* out_dev, uint32_t duration_us, void* stream) {
+    if (!out_dev) return FP8_ERR_NULL;
+    if (duration_us == 0 || duration_us > 100000u) return FP8_ERR_UNSUPPORTED;      // at most a tenth of a second
+    k_sm_clock_probe<<<1, 32, 0, (cudaStream_t)stream>>>(reinterpret_cast<unsigned long long*>(out_dev), (unsigned long long)duration_us * 1000ull);
+    count_launches(1);
+    return launch_status();
 }
 
 const char* fp8_status_string(fp8_status s) {

@@ -85,3 +85,18 @@ def test_self_test_rejects_bad_arguments():
     assert lib.fp8_self_test_expire_wait(1, 3_000_000_000, None) == 5    # longer than about a second
     torch.cuda.synchronize()
     assert api.fp8_async_status() == (0, 0)
+
+
+def test_sm_clock_probe_reports_a_plausible_clock_and_is_bounded():
+    out = torch.zeros(2, dtype=torch.int64, device=DEV)
+    t0 = time.perf_counter()
+    api.fp8_sm_clock_probe(out, 300)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0
+    clocks, ns = (int(v) for v in out.cpu())
+    assert 250_000 <= ns <= 5_000_000, ns                       # about the 300 us asked for
+    mhz = clocks * 1000.0 / ns
+    assert 100.0 < mhz < 3000.0, mhz
+    lib = api.load()
+    assert lib.fp8_sm_clock_probe(None, 100, None) == 1
+    assert lib.fp8_sm_clock_probe(out.data_ptr(), 0, None) == 5 and lib.fp8_sm_clock_probe(out.data_ptr(), 200000, None) == 5
