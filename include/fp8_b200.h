@@ -207,11 +207,10 @@ fp8_status fp8_scale_pow2_from_amax(const float* amax_dev, fp8_format f,
  *                  at K = 49152 on the workloads' tensors, 1.2e-5 at K = 2^20 on heavy-tailed codes); products
  *                  of one sign lose up to (K/32) * 2^-23 of their sum.
  *   FP8_ACC_SPLIT  the accumulator is drained every 2048 of K and the partial sums are added in registers
- *                  with round-to-nearest: below 1e-5 * sum_k|a.b| for any data and any K, at a cost of about a
- *                  tenth of the throughput (measured: 9.6 % at K = 4096, 11.6 % at K = 16384).  Identical to FAST
- *                  for K <= 2048.
+ *                  with round-to-nearest: below 1e-5 * sum_k|a.b| for any data and any K, at a cost of 2.5-4 % of
+ *                  the sustained throughput (measured at K = 4096, 16384 and 49152).  Identical to FAST for K <= 2048.
  *   FAST is the default (acc = 0): zero-mean operands, which is what training tensors are, stay two orders of
- *   magnitude inside the bound at every K of the workloads; a caller whose products share one sign over a long K
+ *   magnitude inside the bound at every K of the workloads; a caller whose products may share one sign over a long K
  *   (K > 2048) should ask for SPLIT.
  * Every GEMM entry point that takes this descriptor honours `acc`; other values give FP8_ERR_ENUM.
  * Reproducibility: a call is bit-reproducible for a given problem (shapes, layouts, data) on a given device.  The

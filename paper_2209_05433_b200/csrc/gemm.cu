@@ -15,7 +15,8 @@
 //                the MMAs into one of two 256-column TMEM accumulators;
 //                tcgen05.commit releases the smem stage in both CTAs / publishes
 //                the finished accumulator to both CTAs' epilogues
-//   warps 2..5   epilogue: tcgen05.ld of the accumulator (each warp owns its 32
+//   warps 2..5   (2..9 for short K, 4..11 for split accumulation)
+//                epilogue: tcgen05.ld of the accumulator (each warp owns its 32
 //                TMEM lanes), multiply by sa_inv*sb_inv, round to bf16 / keep
 //                fp32, amax of the stored values, swizzled staging in shared
 //                memory and TMA tensor stores (edges clipped by the TMA unit).
@@ -317,8 +318,16 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 // accumulator with truncation, so over a long K same-sign products lose up to (K/32) 2^-23 of their sum; here
 // the accumulator is closed every SPLIT_BLOCKS K-blocks and the partial sums are added in registers with
 // round-to-nearest, which keeps the error below 1e-5 of sum|a.b| for any data.
+// Warp layout.  Warp 0 loads, warp 1 issues the MMAs, the epilogue warps start at EPI_BASE.  Split accumulation keeps 128
+// partial sums per epilogue thread and wants two TMEM loads in flight beside them, more registers than a thread of a
+// 320-thread block can have (168): its instances run 12 warps in three aligned groups of four, the first group (loader,
+// MMA issuer, two idle warps) gives registers up with setmaxnreg and the two epilogue groups take them.
+template <bool SPLIT> struct Roles {
+    static constexpr int EPI_BASE = SPLIT ? 4 : 2;
+    static constexpr int REGS_FRONT = 56, REGS_EPILOGUE = 224;   // 4 x 32 x 56 + 8 x 32 x 224 = 64512 <= 65536
+};
 template <int CG, int OUT, int EPI_WARPS, bool SPLIT>
-__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
+__global__ void __launch_bounds__(32 * (Roles<SPLIT>::EPI_BASE + EPI_WARPS), 1)
 k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
            const __grid_constant__ CUtensorMap map_d, const Params p) {
     using G = Geo<CG>;
@@ -372,6 +381,10 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
 
+    constexpr int EPI_BASE = Roles<SPLIT>::EPI_BASE;
+    if (warp < EPI_BASE) {
+    // every warp of the first group executes the same register release, then takes its role
+    if (SPLIT) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Roles<SPLIT>::REGS_FRONT));
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (each CTA loads its own rows)
         uint32_t stage = 0, phase = 0;
@@ -482,17 +495,19 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             }
           }
         }
+    }
     } else {
         // ------------------------------------------------------------ epilogue (each CTA drains its own 128 rows)
+        if (SPLIT) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(Roles<SPLIT>::REGS_EPILOGUE));
         const int q = warp & 3;                                   // TMEM lane quarter this warp may read
         const float sa_inv = __ldg(p.sa_inv);
         const float alpha = p.sb_inv_vec ? 0.0f : sa_inv * __ldg(p.sb_inv);
         const float scale_d = (OUT == OUT_E4M3 || OUT == OUT_E5M2) ? __ldg(p.scale_d) : 1.0f;
         uint32_t running = 0;                                     // bf16: max of stored 16-bit magnitude patterns, two lanes
         float runf = 0.0f;                                        // fp32 / FP8 output: max |v|, NaN once any v is NaN
-        const uint32_t epi_base = ring + RING_BYTES + (uint32_t)(warp - 2) * (uint32_t)EPI_BUFS * EPI_BUF_BYTES;
+        const uint32_t epi_base = ring + RING_BYTES + (uint32_t)(warp - EPI_BASE) * (uint32_t)EPI_BUFS * EPI_BUF_BYTES;
         constexpr int COL_SPLIT = EPI_WARPS / 4;                  // warps sharing a lane quarter split the columns
-        const int col_part = (warp - 2) >> 2;
+        const int col_part = (warp - EPI_BASE) >> 2;
         uint32_t buf = 0;
         const uint64_t stream_out = policy_evict_first();
         bool ok = true;
@@ -521,13 +536,19 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 // not the last chunk of K: move the partial sums into registers (round-to-nearest adds) and
                 // hand the accumulator back
 #pragma unroll
-                for (int s4 = 0; s4 < (SPLIT ? 4 : 0); ++s4) {
-                    uint32_t r[32];
-                    tc_ld32(taddr + col_part * (BN / COL_SPLIT) + s4 * 32, r);
+                for (int s2 = 0; s2 < (SPLIT ? 2 : 0); ++s2) {    // two 32-column loads in flight, one wait for both
+                    uint32_t r[2][32];
+                    tc_ld32(taddr + col_part * (BN / COL_SPLIT) + (2 * s2) * 32, r[0]);
+                    tc_ld32(taddr + col_part * (BN / COL_SPLIT) + (2 * s2 + 1) * 32, r[1]);
                     tc_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        part[(s4 * 32 + i) % (SPLIT ? 128 : 1)] = (have_part ? part[(s4 * 32 + i) % (SPLIT ? 128 : 1)] : 0.0f) + __uint_as_float(r[i]);
+                    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            float& acc_part = part[((2 * s2 + h) * 32 + i) % (SPLIT ? 128 : 1)];
+                            acc_part = (have_part ? acc_part : 0.0f) + __uint_as_float(r[h][i]);
+                        }
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -704,7 +725,7 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
 template <int CG, int OUT, int EPI_WARPS, bool SPLIT = false>
 static fp8_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& md, const Params& p, int64_t num_tiles, cudaStream_t st) {
     auto k = k_gemm_fp8<CG, OUT, EPI_WARPS, SPLIT>;
-    constexpr int THREADS = 64 + 32 * EPI_WARPS;
+    constexpr int THREADS = 32 * (Roles<SPLIT>::EPI_BASE + EPI_WARPS);
     constexpr int MAX_DEVICES = 64;
     static std::mutex mu;
     static int cached_workers[MAX_DEVICES] = {0};                 // 0 = not looked up yet
