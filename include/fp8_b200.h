@@ -99,7 +99,9 @@ fp8_status fp8_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_o
  *   *amax_dev = amax(x); *scale_dev = fmax/amax (same guards); *scale_inv_dev = 1/scale;
  *   out_i = encode_f( binary32(x_i) * scale ).
  * Tensors below 256 MB take ONE kernel, launched cooperatively (all of its blocks resident at once), which
- * crosses one grid-wide barrier between the two passes; the second pass re-reads the tail of x from L2.
+ * crosses one grid-wide barrier between the two passes; the second pass re-reads the tail of x from L2.  A tensor
+ * small enough for the shared memory of the whole GPU (about 33 MB on a B200) is kept there between the passes and
+ * read from global memory only once.
  * Larger tensors (and pointers without 16-byte alignment) take the three streaming kernels back to back on the
  * stream, the conversion walking the tensor from its end, where the amax pass has just been: on long streams
  * that is the faster form, and the workspace is then not touched.

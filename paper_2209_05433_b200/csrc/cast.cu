@@ -422,6 +422,51 @@ __device__ __forceinline__ uint4 ld_v4_policy(const void* ptr, uint64_t policy) 
 }
 
 
+// Grid-wide barrier of the one-launch kernels (all CTAs co-resident), bounded: thread 0 of every CTA announces its
+// arrival in ws[1] and polls until `arrivals` CTAs have, or gives up after `wait_limit` SM clocks (latching the time-out).
+// bcast[0] receives the running amax bits of ws[0], bcast[1] whether the barrier held.  Ends with __syncthreads.
+__device__ __forceinline__ void grid_barrier_read_amax(unsigned int* ws, unsigned int arrivals, long long wait_limit, uint32_t* bcast) {
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&ws[1], 1u);
+        uint32_t okflag = 1u;
+        long long t0 = 0;
+        for (uint32_t spins = 1;; ++spins) {
+            unsigned int arrived;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(arrived) : "l"(&ws[1]) : "memory");
+            if (arrived >= arrivals) break;
+            if ((spins & 255u) == 0u) {
+                const long long now = clock64();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > wait_limit) {
+                    if (atomicCAS(&g_cast_latch[0], 0u, kWaitGridBarrier) == 0u) g_cast_latch[1] = blockIdx.x;
+                    okflag = 0u;
+                    break;
+                }
+            }
+        }
+        unsigned int bits;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(bits) : "l"(&ws[0]) : "memory");
+        bcast[0] = bits;
+        bcast[1] = okflag;
+    }
+    __syncthreads();
+}
+
+// Leaves the control words as they were found: the last CTA out zeroes them (also after a time-out).
+__device__ __forceinline__ void leave_and_reset(unsigned int* ws) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int gone = atomicAdd(&ws[2], 1u);
+        if (gone == gridDim.x - 1) {
+            ws[0] = 0u;
+            ws[2] = 0u;
+            __threadfence();
+            ws[1] = 0u;
+        }
+    }
+}
+
 // Current scaling in ONE launch: amax of x, scale = fmax / amax, quantize with that scale.
 // All CTAs are co-resident (cooperative launch).  ws[0] = running amax bits, ws[1] = arrivals at the
 // grid barrier, ws[2] = departures; the three words are zero on entry and the last CTA to leave puts
@@ -474,31 +519,7 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
     block_atomic_max_bits(m, red, ws);
 
     // ---- grid barrier (bounded), then every CTA reads the same amax
-    if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(&ws[1], 1u);
-        uint32_t okflag = 1u;
-        long long t0 = 0;
-        for (uint32_t spins = 1;; ++spins) {
-            unsigned int arrived;
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(arrived) : "l"(&ws[1]) : "memory");
-            if (arrived >= arrivals) break;
-            if ((spins & 255u) == 0u) {
-                const long long now = clock64();
-                if (t0 == 0) t0 = now;
-                else if (now - t0 > wait_limit) {
-                    if (atomicCAS(&g_cast_latch[0], 0u, kWaitGridBarrier) == 0u) g_cast_latch[1] = blockIdx.x;
-                    okflag = 0u;
-                    break;
-                }
-            }
-        }
-        unsigned int bits;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(bits) : "l"(&ws[0]) : "memory");
-        bcast[0] = bits;
-        bcast[1] = okflag;
-    }
-    __syncthreads();
+    grid_barrier_read_amax(ws, arrivals, wait_limit, bcast);
     const float amax = __uint_as_float(bcast[0]);
     const bool ok = bcast[1] != 0u;
     float scale, scale_inv;
@@ -544,17 +565,67 @@ k_quantize_current(const void* __restrict__ x, size_t n, float fmax, uint8_t* __
         out[i] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * scale, __float_as_uint(xf));
     }
 
-    // ---- leave the workspace as it was found: the last CTA out zeroes it
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int gone = atomicAdd(&ws[2], 1u);
-        if (gone == gridDim.x - 1) {
-            ws[0] = 0u;
-            ws[2] = 0u;
-            __threadfence();
-            ws[1] = 0u;
+    leave_and_reset(ws);
+}
+
+// The same conversion for a tensor that fits the shared memory of the whole GPU (one CTA per SM, each keeping its
+// contiguous slice of x in shared memory between the passes): x is read from global memory ONCE (3 B of traffic per
+// bf16 element instead of 5).  Pass 1 copies the slice into shared memory and folds the amax, the bounded grid barrier
+// follows, pass 2 converts from shared memory.  n is a multiple of the elements per 16-byte item here (the launcher
+// sends ragged sizes elsewhere); ws as in k_quantize_current.
+constexpr int kResidentThreads = 1024;
+template <int WIDE, int FMT, bool NOSAT>
+__global__ void __launch_bounds__(kResidentThreads, 1)
+k_quantize_current_resident(const void* __restrict__ x, size_t n_items, size_t items_per_cta, float fmax, uint8_t* __restrict__ out,
+                            float* amax_out, float* scale_out, float* scale_inv_out, unsigned int* ws,
+                            unsigned int arrivals, long long wait_limit) {
+    extern __shared__ uint4 slice[];
+    __shared__ uint32_t red[32];
+    __shared__ uint32_t bcast[2];
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    const size_t first = (size_t)blockIdx.x * items_per_cta;
+    const size_t mine = first < n_items ? min(items_per_cta, n_items - first) : 0;
+
+    // ---- pass 1: global -> shared, amax on the way (four loads in flight per thread)
+    uint32_t m = 0;
+    size_t i = threadIdx.x;
+    for (; i + 3 * (size_t)kResidentThreads < mine; i += 4 * (size_t)kResidentThreads) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld_in_v4(xv + first + i + (size_t)u * kResidentThreads);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            slice[i + (size_t)u * kResidentThreads] = v[u];
+            m = fold_abs_max<WIDE>(m, v[u]);
         }
     }
+    for (; i < mine; i += kResidentThreads) {
+        const uint4 v = ld_in_v4(xv + first + i);
+        slice[i] = v;
+        m = fold_abs_max<WIDE>(m, v);
+    }
+    block_atomic_max_bits(finish_abs_max<WIDE>(m), red, ws);
+
+    grid_barrier_read_amax(ws, arrivals, wait_limit, bcast);
+    const float amax = __uint_as_float(bcast[0]);
+    const bool ok = bcast[1] != 0u;
+    float scale, scale_inv;
+    scale_pair_from_amax(amax, fmax, scale, scale_inv);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && ok) {
+        *amax_out = amax;
+        *scale_out = scale;
+        *scale_inv_out = scale_inv;
+    }
+
+    // ---- pass 2: shared -> codes (every thread re-reads the items it wrote itself)
+    if (ok) {
+        for (size_t j = threadIdx.x; j < mine; j += kResidentThreads) {
+            const uint4 v = slice[j];
+            if (WIDE == kWideBF16) st_out(reinterpret_cast<uint2*>(out) + first + j, quantize_item_bf16<FMT, NOSAT>(v, scale));
+            else                   st_out(reinterpret_cast<uint32_t*>(out) + first + j, quantize_item_f32<FMT, NOSAT>(v, scale));
+        }
+    }
+    leave_and_reset(ws);
 }
 
 // ---------------------------------------------------------------------------
@@ -1188,6 +1259,45 @@ static fp8_status launch_current(const void* x, size_t n, float fmax, uint8_t* o
     return launch_status();
 }
 
+// Shared memory one CTA may use for its slice (the rest of the 227 KB is the kernel's static arrays and slack).
+constexpr size_t kResidentSliceBytes = 224 * 1024;
+
+template <int WIDE, int FMT, bool NOSAT>
+static fp8_status launch_current_resident(const void* x, size_t n, float fmax, uint8_t* out, float* amax, float* scale, float* scale_inv,
+                                          unsigned int* ws, cudaStream_t st) {
+    constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+    auto k = k_quantize_current_resident<WIDE, FMT, NOSAT>;
+    static std::mutex mu;
+    static bool ready[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FP8_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!ready[dev]) {
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResidentSliceBytes) != cudaSuccess) return FP8_ERR_CUDA;
+            ready[dev] = true;
+        }
+    }
+    size_t n_items = n / EPI;
+    const int sms = sm_count();
+    // whole items per CTA, a multiple of the block size so that pass 1 runs its unrolled loop; no more CTAs than needed
+    size_t items_per_cta = (n_items + (size_t)sms - 1) / (size_t)sms;
+    items_per_cta = (items_per_cta + kResidentThreads - 1) / kResidentThreads * kResidentThreads;
+    int grid = (int)((n_items + items_per_cta - 1) / items_per_cta);
+    if (grid < 1) grid = 1;
+    size_t smem = items_per_cta * 16;
+    unsigned int arrivals = (unsigned int)grid;
+    long long wait_limit = kGridWaitLimitCycles;
+    void* args[] = {(void*)&x, (void*)&n_items, (void*)&items_per_cta, (void*)&fmax, (void*)&out, (void*)&amax, (void*)&scale, (void*)&scale_inv,
+                    (void*)&ws, (void*)&arrivals, (void*)&wait_limit};
+    if (cudaLaunchCooperativeKernel((const void*)k, dim3(grid), dim3(kResidentThreads), args, smem, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return FP8_ERR_UNSUPPORTED;
+    }
+    count_launches(1);
+    return launch_status();
+}
+
 // The vector path needs x 16-byte aligned and out aligned to the codes one item produces; other
 // alignments take the three separate calls (identical results).
 fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_overflow o, uint8_t* out,
@@ -1199,6 +1309,22 @@ fp8_status launch_quantize_current(const void* x, fp8_wide t, size_t n, fp8_form
     const float fmax = f == FP8_E4M3 ? 448.0f : 57344.0f;
     const bool nosat = o == FP8_NOSAT;
     fp8_status s;
+    // a tensor of whole 16-byte items that fits the shared memory of all SMs: read it from global memory once
+    const size_t per_cta = ((n / epi + (size_t)sm_count() - 1) / (size_t)sm_count() + kResidentThreads - 1) / kResidentThreads * kResidentThreads;
+    if (n % epi == 0 && per_cta * 16 <= kResidentSliceBytes) {
+        if (t == FP8_F32) {
+            if (f == FP8_E4M3) s = nosat ? launch_current_resident<kWideF32, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                         : launch_current_resident<kWideF32, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+            else               s = nosat ? launch_current_resident<kWideF32, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                         : launch_current_resident<kWideF32, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+        } else {
+            if (f == FP8_E4M3) s = nosat ? launch_current_resident<kWideBF16, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                         : launch_current_resident<kWideBF16, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+            else               s = nosat ? launch_current_resident<kWideBF16, kE5M2, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
+                                         : launch_current_resident<kWideBF16, kE5M2, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
+        }
+        if (s != FP8_ERR_UNSUPPORTED) return s;                   // refused (e.g. not all CTAs can be resident): the general kernel below
+    }
     if (t == FP8_F32) {
         if (f == FP8_E4M3) s = nosat ? launch_current<kWideF32, kE4M3, true>(x, n, fmax, out, amax, scale, scale_inv, ws, st)
                                      : launch_current<kWideF32, kE4M3, false>(x, n, fmax, out, amax, scale, scale_inv, ws, st);
