@@ -155,18 +155,20 @@ __device__ __forceinline__ uint32_t quantize_item_f32(const uint4& v, float scal
 // ---------------------------------------------------------------------------
 
 // One word set to zero: the start value of an amax accumulated with atomicMax by the kernel launched next.
-// It waits for everything earlier in the stream first, so the kernel behind it may read its inputs at once.
+// It lets that kernel be scheduled at once (so its launch overlaps this kernel's wait for everything earlier in the
+// stream), then waits, then writes; the kernel behind it waits for this one before it touches memory.
 __global__ void k_zero_word(uint32_t* p) {
+    grid_launch_dependents();
     grid_dependency_wait();
     *p = 0u;
 }
 
-// amax over n elements.  Launched behind k_zero_word(amax_bits): the loads start while that kernel runs, only the
-// final atomicMax waits for it.
+// amax over n elements.  Launched behind k_zero_word(amax_bits), which has zeroed the accumulator.
 template <int WIDE, int UNROLL>
 __global__ void __launch_bounds__(kThreads) k_amax(const void* __restrict__ x, size_t n, uint32_t* amax_bits) {
     __shared__ uint32_t red[32];
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;              // elements per 16-byte item
+    grid_dependency_wait();
     const uint4* xv = reinterpret_cast<const uint4*>(x);
     const size_t n_items = n / EPI;
     const size_t per_chunk = (size_t)kThreads * UNROLL;
@@ -192,19 +194,17 @@ __global__ void __launch_bounds__(kThreads) k_amax(const void* __restrict__ x, s
     if (blockIdx.x == 0 && threadIdx.x < n - n_items * EPI)      // ragged tail, fewer than EPI elements
         m = max(m, canonical_nan_bits(scalar_abs_bits<WIDE>(x, n_items * EPI + threadIdx.x)));
     grid_launch_dependents();
-    grid_dependency_wait();                                      // the accumulator has been zeroed
     block_atomic_max_bits(m, red, amax_bits);
 }
 
-// quantize n elements (+ optional amax of the input in the same pass).  With amax the kernel is launched behind
-// k_zero_word and waits only before its atomicMax; without, it waits before its first load.
+// quantize n elements (+ optional amax of the input in the same pass; the kernel is then launched behind k_zero_word).
 template <int WIDE, int FMT, bool NOSAT, bool WITH_AMAX, int UNROLL>
 __global__ void __launch_bounds__(kThreads)
 k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale_dev,
            uint8_t* __restrict__ out, uint32_t* amax_bits, int reverse) {
     __shared__ uint32_t red[32];
     constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
-    if (!WITH_AMAX) grid_dependency_wait();
+    grid_dependency_wait();
     const float scale = *scale_dev;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
     const size_t n_items = n / EPI;
@@ -245,10 +245,7 @@ k_quantize(const void* __restrict__ x, size_t n, const float* __restrict__ scale
         out[i] = (uint8_t)encode_scaled<FMT, NOSAT>(xf * scale, __float_as_uint(xf));
     }
     grid_launch_dependents();
-    if (WITH_AMAX) {
-        grid_dependency_wait();                                  // the accumulator has been zeroed
-        block_atomic_max_bits(finish_abs_max<WIDE>(m), red, amax_bits);
-    }
+    if (WITH_AMAX) block_atomic_max_bits(finish_abs_max<WIDE>(m), red, amax_bits);
 }
 
 // dequantize: 8 codes (bf16 out) or 4 codes (f32 out) per item, one 16-byte store each.
@@ -1231,7 +1228,7 @@ static fp8_status launch_dequantize(const uint8_t* c, size_t n, const float* si,
 }
 
 // The start value of an amax: a one-thread kernel rather than a memset node, so that the kernel behind it can be
-// scheduled, and read its inputs, while this one runs.
+// scheduled while this one still waits for the stream's earlier work.
 static fp8_status zero_word(void* p, cudaStream_t st) {
     if (launch_programmatic(k_zero_word, dim3(1), dim3(1), st, reinterpret_cast<uint32_t*>(p)) != cudaSuccess) return FP8_ERR_CUDA;
     count_launches(1);
