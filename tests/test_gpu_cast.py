@@ -261,7 +261,7 @@ def test_config2_large_sizes_sampled(log2n):
 # ------------------------------------------ fused current scaling (one launch) --
 
 @pytest.mark.parametrize("wide", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("n", [0, 1, 7, 8, 9, 1000, 4099, (1 << 20) + 3, (1 << 24) + 17])
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 9, 1000, 4099, 1 << 20, (1 << 20) + 3, 1 << 22, (1 << 24) + 17])
 def test_quantize_current_equals_three_calls_and_oracle(wide, n):
     x = synth.activations(n, 3, dtype=wide, device=DEV)
     x_np = to_np_bits(x)
@@ -280,6 +280,33 @@ def test_quantize_current_equals_three_calls_and_oracle(wide, n):
             _assert_codes(out[:n].cpu().numpy(), oracle.quantize(x_np, ws, fmt, overflow, threads=THREADS), x_np)
             assert bool((out[n:] == 0xA5).all())
             assert bool((api.current_scaling_workspace(x.device) == 0).all())
+
+
+@pytest.mark.parametrize("wide", [torch.float32, torch.bfloat16])
+def test_quantize_current_at_the_shared_memory_capacity(wide):
+    """the largest tensor the shared-memory-resident kernel takes (every SM's slice full), one item more (the general
+    one-launch kernel), and the largest with a NaN in the last slice: same amax, scales and codes as the oracle"""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    epi = 8 if wide == torch.bfloat16 else 4
+    full = sms * 14336 * epi                                   # 224 KB of 16-byte items per SM
+    for n, poke in ((full, None), (full + epi, None), (full, float("nan")), (full - 1024 * epi * 3, float("inf"))):
+        x = synth.normal_laplace_mixture(n, 13, synth.T_ID, dtype=wide, device=DEV)
+        if poke is not None:
+            x[n - 5] = poke
+        x_np = to_np_bits(x)
+        a, s, si = _scalar(-1.0), _scalar(-1.0), _scalar(-1.0)
+        out = torch.full((n + 64,), 0xA5, dtype=torch.uint8, device=DEV)
+        api.fp8_quantize_current(x, api.E5M2, out[:n], a, s, si)
+        torch.cuda.synchronize()
+        assert api.fp8_async_status()[0] == 0
+        want_bits = oracle.amax_bits(x_np, THREADS)
+        ws, wsi = oracle.scale_from_amax(np.array([want_bits], dtype=np.uint32).view(np.float32)[0], oracle.E5M2)
+        assert a.cpu().numpy().view(np.uint32)[0] == want_bits and s.item() == ws and si.item() == wsi
+        _assert_codes(out[:n].cpu().numpy(), oracle.quantize(x_np, ws, oracle.E5M2, threads=THREADS), x_np)
+        assert bool((out[n:] == 0xA5).all())
+        assert bool((api.current_scaling_workspace(x.device) == 0).all())
+        del x, out
+    torch.cuda.empty_cache()
 
 
 def test_quantize_current_specials_and_unaligned():

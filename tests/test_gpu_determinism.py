@@ -66,3 +66,35 @@ def test_batched_gemm_and_casts_are_bitwise_repeatable():
     _repeat(lambda: api.fp8_quantize_current(x, api.E5M2, o, sc[0:1], sc[1:2], sc[2:3]), o, 150)
     back = torch.empty_like(x)
     _repeat(lambda: api.fp8_fake_quantize(x, api.E4M3, s3, sc[2:3], back), back, 100)
+
+
+def test_back_to_back_dependent_casts_see_each_others_results():
+    """The cast kernels are launched with programmatic stream serialization (a kernel may be scheduled while its
+    predecessor drains).  Chains in which every kernel consumes what the one before it wrote, enqueued without any
+    host synchronisation and with buffers that are overwritten from one round to the next, must give the results of
+    strictly serial execution: codes -> dequantize equals the one-pass simulated conversion, round after round."""
+    import numpy as np
+    from paper_2209_05433_b200 import synth
+    dev = "cuda"
+    sizes = [(1 << 12) + 8, 1 << 16, (1 << 20) + 16, 1 << 22, (1 << 23) + 24]
+    xs = [synth.normal_laplace_mixture(n, 31 + i, synth.T_ID, dtype=torch.bfloat16, device=dev) for i, n in enumerate(sizes)]
+    nmax = max(sizes)
+    codes = torch.empty(nmax, dtype=torch.uint8, device=dev)          # shared scratch, rewritten by every round
+    back = torch.empty(nmax, dtype=torch.bfloat16, device=dev)
+    direct = torch.empty(nmax, dtype=torch.bfloat16, device=dev)
+    sc = torch.zeros(3, dtype=torch.float32, device=dev)
+    a, s, si = sc[0:1], sc[1:2], sc[2:3]
+    bad = torch.zeros(1, dtype=torch.int64, device=dev)
+    for rnd in range(40):
+        for x in xs:
+            n = x.numel()
+            fmt = api.E4M3 if rnd & 1 else api.E5M2
+            api.fp8_amax(x, a)                                        # zeroing kernel + reduction
+            api.fp8_scale_from_amax(a, fmt, s, si)                    # reads the amax
+            api.fp8_quantize(x, fmt, s, codes[:n])                    # reads the scale
+            api.fp8_dequantize(codes[:n], fmt, si, back[:n])          # reads the codes and the inverse scale
+            api.fp8_fake_quantize(x, fmt, s, si, direct[:n])          # the same arithmetic in one pass
+            bad += (back[:n].view(torch.int16) != direct[:n].view(torch.int16)).sum()
+    torch.cuda.synchronize()
+    assert api.fp8_async_status()[0] == 0
+    assert int(bad.item()) == 0
