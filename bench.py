@@ -746,6 +746,8 @@ def run_ours(args, world, rank, local):
             "regime": "sustained: per-launch CUDA events inside a loop of %d whole steps (%.2f s), divided by 2 x %s bf16 sustained cuBLAS "
                       "TFLOP/s (fp8:bf16 nominal ratio 2)" % (n_sus, sus_ms / 1e3, pk["source"]),
             "algorithmic_flops_per_launch": step.flops_per_gemm,
+            "accumulation": "library default: partial sums every 2048 of K added in registers (1e-5 * sum|a.b| for any data); "
+                            "the single-accumulator mode FP8_ACC_FAST is 2.5-4 % faster, see next_rows",
             "per_gemm_tflops": sus["gemm_tflops"],
             "clock_normalised": {"sm_mhz_on_device_median": round(device_mhz_median, 1) if device_mhz_median else None,
                                  "frac_of_tensor_pipe_rate": clock_normalised(a_sus, device_mhz_median),

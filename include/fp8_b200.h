@@ -49,7 +49,7 @@ typedef enum { FP8_SATURATE = 0, FP8_NOSAT = 1 } fp8_overflow;
 /* Which index of a GEMM operand is contiguous in memory. */
 typedef enum { FP8_MAJOR_K = 0, FP8_MAJOR_MN = 1 } fp8_major;
 /* how a GEMM accumulates over K (see fp8_gemm) */
-typedef enum { FP8_ACC_FAST = 0, FP8_ACC_SPLIT = 1 } fp8_accumulate;
+typedef enum { FP8_ACC_SPLIT = 0, FP8_ACC_FAST = 1 } fp8_accumulate;
 
 /*
  * fp8_amax — maximum magnitude of a tensor (Section 2: the quantity the scale
@@ -204,16 +204,14 @@ fp8_status fp8_scale_pow2_from_amax(const float* amax_dev, fp8_format f,
  * (amax = 0); K == 0 writes zeros.
  * Accumulation (`acc`): the products are exact and the tensor core adds them, 32 of K at a time, into a
  * binary32 accumulator whose additions round toward zero.
- *   FP8_ACC_FAST   one accumulator over all of K.  The error is below 1e-5 * sum_k|a.b| for K <= 2048 on any
- *                  data; on products of mixed sign (training tensors) it grows slowly with K (measured 1.4e-7
- *                  at K = 49152 on the workloads' tensors, 1.2e-5 at K = 2^20 on heavy-tailed codes); products
- *                  of one sign lose up to (K/32) * 2^-23 of their sum.
- *   FP8_ACC_SPLIT  the accumulator is drained every 2048 of K and the partial sums are added in registers
- *                  with round-to-nearest: below 1e-5 * sum_k|a.b| for any data and any K, at a cost of 2.5-4 % of
- *                  the sustained throughput (measured at K = 4096, 16384 and 49152).  Identical to FAST for K <= 2048.
- *   FAST is the default (acc = 0): zero-mean operands, which is what training tensors are, stay two orders of
- *   magnitude inside the bound at every K of the workloads; a caller whose products may share one sign over a long K
- *   (K > 2048) should ask for SPLIT.
+ *   FP8_ACC_SPLIT  (0, the default of a zero-initialised descriptor) the accumulator is drained every 2048 of K and the
+ *                  partial sums are added in registers with round-to-nearest: below 1e-5 * sum_k|a.b| for ANY data and
+ *                  any K.  For K <= 2048 it is the single accumulator.
+ *   FP8_ACC_FAST   one accumulator over all of K, 2.5-4 % faster at K = 4096 .. 49152.  The error is below
+ *                  1e-5 * sum_k|a.b| for K <= 2048 on any data; on products of mixed sign (training tensors: zero-mean
+ *                  weights and gradients) it grows slowly with K (measured 1.4e-7 at K = 49152 on the workloads'
+ *                  tensors, 1.2e-5 at K = 2^20 on heavy-tailed codes); products that all share one sign lose up to
+ *                  (K/32) * 2^-23 of their sum (measured 3.7-5.3e-5 at K = 49152).  For callers who know their operands.
  * Every GEMM entry point that takes this descriptor honours `acc`; other values give FP8_ERR_ENUM.
  * Reproducibility: a call is bit-reproducible for a given problem (shapes, layouts, data) on a given device.  The
  * order in which the K-blocks of an output tile are accumulated (from the start or from the end of K) depends on

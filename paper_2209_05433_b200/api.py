@@ -18,7 +18,7 @@ E4M3, E5M2 = 0, 1            # fp8_format
 F32, BF16 = 0, 1             # fp8_wide
 SATURATE, NOSAT = 0, 1       # fp8_overflow
 MAJOR_K, MAJOR_MN = 0, 1     # fp8_major
-ACC_FAST, ACC_SPLIT = 0, 1    # fp8_accumulate
+ACC_SPLIT, ACC_FAST = 0, 1    # fp8_accumulate: bounded error for any data (default) / one accumulator
 
 EXPORTS = ["fp8_amax", "fp8_scale_from_amax", "fp8_quantize", "fp8_quantize_current",
            "fp8_quantize_current_workspace_bytes", "fp8_quantize_current_static", "fp8_dequantize", "fp8_fake_quantize",
@@ -225,14 +225,14 @@ def fp8_scale_pow2_from_amax(amax: torch.Tensor, fmt: int, scale_out: torch.Tens
 
 def fp8_gemm(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
              scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, amax_out: torch.Tensor | None = None,
-             acc: int = ACC_FAST) -> None:
+             acc: int = ACC_SPLIT) -> None:
     """D[M,N] = (A[M,K] . B[K,N]) * scale_inv_a * scale_inv_b.
 
     A is a 2-D uint8 tensor stored [M,K] when ``ma == MAJOR_K`` or [K,M] when
     ``ma == MAJOR_MN``; B is stored [N,K] when ``mb == MAJOR_K`` or [K,N] when
     ``mb == MAJOR_MN``.  Row pitches are taken from the tensors' strides.
-    ``acc`` selects one accumulator over all of K (ACC_FAST) or partial sums every 2048 of K added in
-    registers (ACC_SPLIT: tolerance met on same-sign data at any K)."""
+    ``acc``: ACC_SPLIT (default) adds partial sums every 2048 of K in registers (tolerance met on any data at any
+    K); ACC_FAST keeps one accumulator over all of K (a few per cent faster; for zero-mean operands)."""
     d = _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc)
     _check(load().fp8_gemm(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
                            _scalar(scale_inv_a, "scale_inv_a"), _scalar(scale_inv_b, "scale_inv_b"),
@@ -263,7 +263,7 @@ def fp8_gemm_splitk_workspace(M: int, N: int, K: int) -> tuple[int, int]:
 
 def fp8_gemm_splitk(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
                     scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, workspace: torch.Tensor | None,
-                    amax_out: torch.Tensor | None = None, acc: int = ACC_FAST) -> None:
+                    amax_out: torch.Tensor | None = None, acc: int = ACC_SPLIT) -> None:
     """fp8_gemm with the contraction cut into slices when the problem has few output tiles; ``workspace`` is a
     CUDA tensor of at least fp8_gemm_splitk_workspace(M, N, K)[1] bytes (None when that is 0)."""
     d = _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc)
@@ -276,7 +276,7 @@ def fp8_gemm_splitk(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int,
 
 def fp8_gemm_fp8out(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor, fd: int,
                     scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, scale_d: torch.Tensor,
-                    amax_out: torch.Tensor | None = None, overflow: int = SATURATE, acc: int = ACC_FAST) -> None:
+                    amax_out: torch.Tensor | None = None, overflow: int = SATURATE, acc: int = ACC_SPLIT) -> None:
     """D[M,N] (uint8 codes of format fd) = encode((A . B) * scale_inv_a * scale_inv_b * scale_d); amax_out
     receives the amax of the result before the output scale and conversion.  Layout rules as fp8_gemm."""
     d = _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc, codes_out=True)
@@ -341,7 +341,7 @@ def fp8_quantize_transpose(x: torch.Tensor, fmt: int, scale: torch.Tensor, out: 
 
 def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
                             scale_inv_a: torch.Tensor, scale_inv_b_vec: torch.Tensor, amax_out: torch.Tensor | None = None,
-                            acc: int = ACC_FAST) -> None:
+                            acc: int = ACC_SPLIT) -> None:
     """fp8_gemm with one inverse scale per column of B (per output channel)."""
     d = _gemm_desc_2d(A, ma, B, mb, D, fa, fb, acc)
     _check(load().fp8_gemm_channel_scales(ctypes.byref(d), A.data_ptr(), B.data_ptr(), D.data_ptr(),
@@ -352,7 +352,7 @@ def fp8_gemm_channel_scales(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, 
 
 def fp8_gemm_batched(A: torch.Tensor, fa: int, ma: int, B: torch.Tensor, fb: int, mb: int, D: torch.Tensor,
                      scale_inv_a: torch.Tensor, scale_inv_b: torch.Tensor, amax_out: torch.Tensor | None = None,
-                     acc: int = ACC_FAST) -> None:
+                     acc: int = ACC_SPLIT) -> None:
     """Batched fp8_gemm: A, B are 3-D uint8 tensors [batch, rows, cols] (layouts per member as fp8_gemm), D is
     [batch, M, N]; the batch strides are taken from the tensors."""
     if A.dtype != torch.uint8 or B.dtype != torch.uint8 or A.dim() != 3 or B.dim() != 3 or D.dim() != 3:

@@ -115,9 +115,9 @@ def _linear_layer(seed, T, I, O, w_sigma, passes, n_random):
         Y = torch.empty(T, O, dtype=torch.bfloat16, device=DEV)
         api.fp8_gemm(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, six, siw, amax)
         _check_gemm(Y, amax, Xh, E4, (I, 1), Wh, E4, (O, 1), I, wsix, wsiw, rng, "fprop K=%d" % I, n_random)
-        # the same product with split accumulation (partial sums every 2048 of K added in registers)
-        api.fp8_gemm(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, six, siw, amax, acc=api.ACC_SPLIT)
-        _check_gemm(Y, amax, Xh, E4, (I, 1), Wh, E4, (O, 1), I, wsix, wsiw, rng, "fprop K=%d split accumulation" % I, n_random // 8, 4)
+        # the same product with one accumulator over all of K (FP8_ACC_FAST; the default adds partial sums every 2048 of K)
+        api.fp8_gemm(Xq, api.E4M3, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_MN, Y, six, siw, amax, acc=api.ACC_FAST)
+        _check_gemm(Y, amax, Xh, E4, (I, 1), Wh, E4, (O, 1), I, wsix, wsiw, rng, "fprop K=%d one accumulator" % I, n_random // 8, 4)
         del Y
     if "dgrad" in passes or "wgrad" in passes:
         dY = synth.gradients(T * O, seed, device=DEV).view(T, O)
@@ -129,16 +129,16 @@ def _linear_layer(seed, T, I, O, w_sigma, passes, n_random):
             api.fp8_gemm(Gq, api.E5M2, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, sig, siw, amax)
             step = 4 if O > 16384 else 1                  # K = 49152: every fourth row of the two whole tiles
             _check_gemm(dX, amax, Gh, E5, (O, 1), Wh, E4, (1, O), O, wsig, wsiw, rng, "dgrad K=%d" % O, n_random, step)
-            # the same product with split accumulation (partial sums every 2048 of K added in registers)
-            api.fp8_gemm(Gq, api.E5M2, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, sig, siw, amax, acc=api.ACC_SPLIT)
-            _check_gemm(dX, amax, Gh, E5, (O, 1), Wh, E4, (1, O), O, wsig, wsiw, rng, "dgrad K=%d split accumulation" % O, n_random // 4, 4 * step)
+            # the same product with one accumulator over all of K (FP8_ACC_FAST; the default adds partial sums every 2048 of K)
+            api.fp8_gemm(Gq, api.E5M2, api.MAJOR_K, Wq, api.E4M3, api.MAJOR_K, dX, sig, siw, amax, acc=api.ACC_FAST)
+            _check_gemm(dX, amax, Gh, E5, (O, 1), Wh, E4, (1, O), O, wsig, wsiw, rng, "dgrad K=%d one accumulator" % O, n_random // 4, 4 * step)
             del dX
         if "wgrad" in passes:    # dW[I,O] = X^T . dY
             dW = torch.empty(I, O, dtype=torch.bfloat16, device=DEV)
             api.fp8_gemm(Xq, api.E4M3, api.MAJOR_MN, Gq, api.E5M2, api.MAJOR_MN, dW, six, sig, amax)
             _check_gemm(dW, amax, Xh, E4, (1, I), Gh, E5, (O, 1), T, wsix, wsig, rng, "wgrad K=%d" % T, n_random)
-            api.fp8_gemm(Xq, api.E4M3, api.MAJOR_MN, Gq, api.E5M2, api.MAJOR_MN, dW, six, sig, amax, acc=api.ACC_SPLIT)
-            _check_gemm(dW, amax, Xh, E4, (1, I), Gh, E5, (O, 1), T, wsix, wsig, rng, "wgrad K=%d split accumulation" % T, n_random // 8, 4)
+            api.fp8_gemm(Xq, api.E4M3, api.MAJOR_MN, Gq, api.E5M2, api.MAJOR_MN, dW, six, sig, amax, acc=api.ACC_FAST)
+            _check_gemm(dW, amax, Xh, E4, (1, I), Gh, E5, (O, 1), T, wsix, wsig, rng, "wgrad K=%d one accumulator" % T, n_random // 8, 4)
             del dW
     torch.cuda.empty_cache()
 
