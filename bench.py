@@ -144,8 +144,9 @@ class ClockSampler:
 class LinearStep:
     """Buffers and call sequence of one step.  Everything the step computes runs in the library's kernels."""
 
-    def __init__(self, torch, api, synth, device, layer, seed_offset=0):
+    def __init__(self, torch, api, synth, device, layer, seed_offset=0, acc=None):
         L = LAYERS[layer]
+        self.acc = api.ACC_SPLIT if acc is None else acc          # accumulation mode of the GEMMs (library default)
         self.torch, self.api, self.layer = torch, api, layer
         self.T, self.I, self.O, self.passes = L["tokens"], L["d_in"], L["d_out"], L["passes"]
         T, I, O, seed = self.T, self.I, self.O, L["seed"] + seed_offset
@@ -184,11 +185,11 @@ class LinearStep:
             ("dequantize", lambda: a.fp8_dequantize(self.Xq, E4, self.six, self.Xhat)),
         ]
         if "fprop" in self.passes:      # Y[T,O] = X[T,I] . W[I,O]   (W stored with the output index contiguous)
-            calls.append(("gemm_fprop", lambda: a.fp8_gemm(self.Xq, E4, KM, self.Wq, E4, MN, self.Y, self.six, self.siw, self.ay)))
+            calls.append(("gemm_fprop", lambda: a.fp8_gemm(self.Xq, E4, KM, self.Wq, E4, MN, self.Y, self.six, self.siw, self.ay, acc=self.acc)))
         if "dgrad" in self.passes:      # dX[T,I] = dY[T,O] . W^T      (W stored [I,O] is the [N,K] layout here)
-            calls.append(("gemm_dgrad", lambda: a.fp8_gemm(self.dYq, E5, KM, self.Wq, E4, KM, self.dX, self.sig, self.siw, self.adx)))
+            calls.append(("gemm_dgrad", lambda: a.fp8_gemm(self.dYq, E5, KM, self.Wq, E4, KM, self.dX, self.sig, self.siw, self.adx, acc=self.acc)))
         if "wgrad" in self.passes:      # dW[I,O] = X^T . dY           (both operands stored with the contraction index outermost)
-            calls.append(("gemm_wgrad", lambda: a.fp8_gemm(self.Xq, E4, MN, self.dYq, E5, MN, self.dW, self.six, self.sig, self.adw)))
+            calls.append(("gemm_wgrad", lambda: a.fp8_gemm(self.Xq, E4, MN, self.dYq, E5, MN, self.dW, self.six, self.sig, self.adw, acc=self.acc)))
         return calls
 
     def cast_elements(self, label):
@@ -549,7 +550,7 @@ def run_reference(args, world, rank):
 def run_only(args, torch, api, synth, device):
     """One call of a layer's step, alone (what the ncu captures under profiles/ run): a full step first to set
     scales and codes, then `--steps` launches of the named call."""
-    step = LinearStep(torch, api, synth, device, args.layer)
+    step = LinearStep(torch, api, synth, device, args.layer, acc=api.ACC_FAST if args.acc == "fast" else api.ACC_SPLIT)
     step.run()
     for _ in range(max(args.warmup, 1)):
         step.run(args.only)
@@ -850,6 +851,7 @@ def main():
     ap.add_argument("--config", type=int, default=0, help="run one of the five named workloads (1..5), every call timed alone")
     ap.add_argument("--only", default=None, help="time only the calls with this label of a layer's step (e.g. gemm_fprop, quantize_current_W)")
     ap.add_argument("--layer", choices=sorted(LAYERS), default=HEADLINE, help="layer of --only")
+    ap.add_argument("--acc", choices=["split", "fast"], default="split", help="accumulation mode of the GEMMs under --only (split = library default)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         spawn_ranks(args.gpus)
