@@ -531,10 +531,11 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
             constexpr int SUBS = CHUNK / 32;                      // 32-column TMEM loads per box
             constexpr int WORDS = 32 * ESZ / 4;                   // 32-bit words one load contributes to the row
             constexpr int NBOX = BN / CHUNK / COL_SPLIT;          // boxes per warp and tile
-            const bool have_part = SPLIT && kc != 0;
-            if (SPLIT && kc + chunk_blocks < k_pad) {
-                // not the last chunk of K: move the partial sums into registers (round-to-nearest adds) and
-                // hand the accumulator back
+            if (SPLIT) {
+                // Split accumulation: every chunk of K, the last one included, is first moved into registers
+                // (round-to-nearest adds onto the partial sums) and the accumulator handed back at once, so that
+                // the MMA warp never waits for the conversion and the stores of a tile's last chunk.
+                const bool have_part = kc != 0;
 #pragma unroll
                 for (int s2 = 0; s2 < (SPLIT ? 2 : 0); ++s2) {    // two 32-column loads in flight, one wait for both
                     uint32_t r[2][32];
@@ -556,7 +557,7 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                     if (CG == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0));
                     else         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
                 }
-                continue;
+                if (kc + chunk_blocks < k_pad) continue;          // more of K to come
             }
 #pragma unroll (SPLIT ? NBOX : 1)
             for (int cc = 0; cc < NBOX; ++cc) {
@@ -576,16 +577,15 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 uint32_t rr[PRE][32];
 #pragma unroll
                 for (int sub = 0; sub < SUBS; ++sub) {
-                    if (sub % PRE == 0) {
+                    if (!SPLIT && sub % PRE == 0) {
 #pragma unroll
                         for (int g = 0; g < PRE; ++g) tc_ld32(taddr + c * CHUNK + (sub + g) * 32, rr[g]);
                         tc_wait_ld();
                     }
                     uint32_t (&r)[32] = rr[sub % PRE];
-                    if (have_part) {
+                    if (SPLIT) {                                  // the sums are in registers already
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            r[i] = __float_as_uint(__uint_as_float(r[i]) + part[((cc * SUBS + sub) * 32 + i) % (SPLIT ? 128 : 1)]);
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(part[((cc * SUBS + sub) * 32 + i) % (SPLIT ? 128 : 1)]);
                     }
                     float v[32];
                     if (p.sb_inv_vec) {                       // per-channel weight scales: one alpha per column
@@ -659,11 +659,13 @@ k_gemm_fp8(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CU
                 }
                 buf = (buf + 1u) % (uint32_t)EPI_BUFS;
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {                                      // accumulator may be overwritten: tell the leader's MMA warp
-                if (CG == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0));
-                else         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
+            if (!SPLIT) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {                                  // accumulator may be overwritten: tell the leader's MMA warp
+                    if (CG == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0));
+                    else         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
+                }
             }
           }
         }
