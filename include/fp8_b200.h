@@ -93,7 +93,7 @@ fp8_status fp8_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, fp8_o
                         const float* scale_dev, uint8_t* out, float* amax_dev, void* stream);
 
 /*
- * fp8_quantize_current — Section 2, the whole "current scaling" conversion of one tensor in ONE call:
+ * fp8_quantize_current — Section 2, the whole current-scaling conversion of one tensor in ONE call:
  * the scale is chosen from the tensor's own maximum magnitude, then the tensor is converted with it.
  * Results are identical, bit for bit, to fp8_amax + fp8_scale_from_amax + fp8_quantize:
  *   *amax_dev = amax(x); *scale_dev = fmax/amax (same guards); *scale_inv_dev = 1/scale;
@@ -163,7 +163,7 @@ fp8_status fp8_dequantize(const uint8_t* c, size_t n, fp8_format f,
                           const float* scale_inv_dev, void* out, fp8_wide t, void* stream);
 
 /*
- * fp8_fake_quantize — Section 4: the paper's own experiments ran "simulated FP8": tensors were converted
+ * fp8_fake_quantize — Section 4: the paper's own experiments simulated FP8: tensors were converted
  * to FP8 (scale factor, rounding and saturation included) and straight back to the wider type, and the
  * arithmetic stayed in that wider type.  This is that round trip in one pass over the tensor:
  *   out_i = round_t( decode_f( encode_f( binary32(x_i) * scale ) ) * scale_inv ),  out has the type of x.
@@ -174,8 +174,8 @@ fp8_status fp8_fake_quantize(const void* x, fp8_wide t, size_t n, fp8_format f, 
                              const float* scale_dev, const float* scale_inv_dev, void* out, void* stream);
 
 /*
- * fp8_scale_pow2_from_amax — Section 3.2: a programmable exponent bias "is equivalent to allowing only
- * powers of 2 as scaling factors".  scale = the largest power of two not above fmax/amax (same guards
+ * fp8_scale_pow2_from_amax — Section 3.2: a programmable exponent bias amounts to restricting the scale
+ * factors to powers of two.  scale = the largest power of two not above fmax/amax (same guards
  * as fp8_scale_from_amax), scale_inv = 1/scale (exact).  Converting with this scale is converting to an
  * E4M3/E5M2 variant whose exponent bias is shifted by log2(scale) (the bias sweep of Section 4.3).
  */
@@ -232,8 +232,8 @@ fp8_status fp8_gemm(const fp8_gemm_desc* d, const uint8_t* A, const uint8_t* B, 
                     float* amax_d_dev, void* stream);
 
 /*
- * fp8_gemm_fp8out — Section 2: operations on FP8 inputs produce higher-precision results, "optionally
- * converting the results to FP8 prior to writing them to memory".  Same contraction as fp8_gemm, but the
+ * fp8_gemm_fp8out — Section 2: operations on FP8 inputs produce higher-precision results, which may
+ * be converted to FP8 before they are written to memory.  Same contraction as fp8_gemm, but the
  * epilogue converts instead of storing a wide value:
  *   v[i,j] = (sum_k decode_fa(A[i,k]) * decode_fb(B[k,j])) * (sa_inv * sb_inv)      (binary32)
  *   D[i,j] = encode_fd( v[i,j] * scale_d )       conversion rules of fp8_quantize (RNE, specials, `od`)
@@ -270,8 +270,8 @@ fp8_status fp8_quantize_transpose(const void* x, fp8_wide t, int64_t rows, int64
                                   float* amax_dev, void* stream);
 
 /*
- * Per-channel scale factors — Section 4.2: post-training quantization uses "per-channel scaling factors for
- * weights, per-tensor scaling factors for activations".  A channel is a row or a column of a 2-D tensor
+ * Per-channel scale factors — Section 4.2: post-training quantization scales weights channel by channel and
+ * activations with one factor per tensor.  A channel is a row or a column of a 2-D tensor
  * x (rows x cols, row-major, pitch ld elements): axis 0 = one channel per column, axis 1 = one per row.
  *
  * fp8_amax_channels      amax_vec[c] = amax over channel c (definition of fp8_amax), OVERWRITTEN.
@@ -301,8 +301,8 @@ fp8_status fp8_gemm_channel_scales(const fp8_gemm_desc* d, const uint8_t* A, con
                                    float* amax_d_dev, void* stream);
 
 /*
- * fp8_gemm_batched — Section 4.2 quantizes "all input tensors to matrix-multiply operations (including
- * attention batched matrix multiplies)".  `batch` independent products with the same shape, layouts,
+ * fp8_gemm_batched — Section 4.2 quantizes the inputs of every matrix multiply, the batched
+ * products of attention among them.  `batch` independent products with the same shape, layouts,
  * formats and per-tensor scales (one scale for the whole batched tensor), in one launch:
  *   D_b = (A_b . B_b) * (sa_inv * sb_inv),   A_b = A + b*stride_a, B_b = B + b*stride_b, D_b = D + b*stride_d
  * Strides are in elements of the respective tensor and 16-byte aligned (in bytes).  The members of D lie at

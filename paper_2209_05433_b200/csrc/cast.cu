@@ -626,7 +626,7 @@ k_quantize_current_resident(const void* __restrict__ x, size_t n_items, size_t i
 }
 
 // ---------------------------------------------------------------------------
-// fake quantization: wide -> FP8 -> wide in one pass (what "simulated FP8" runs, Section 4)
+// fake quantization: wide -> FP8 -> wide in one pass (what the simulated-FP8 experiments of Section 4 run)
 // ---------------------------------------------------------------------------
 
 // one scaled value -> its FP8 code -> back to binary32 times scale_inv (scalar path, any input)
@@ -704,7 +704,7 @@ k_fake_quantize_elementwise(const void* __restrict__ x, size_t n, const float* _
 }
 
 // power-of-two scale: the largest power of two not above fmax / amax (same guards as k_scale_from_amax).
-// With such a scale the conversion is the paper's "programmable exponent bias" variant (Section 3.2).
+// With such a scale the conversion is the paper's variant with a programmable exponent bias (Section 3.2).
 __global__ void k_scale_pow2_from_amax(const float* amax_dev, float fmax, float* scale_dev, float* scale_inv_dev) {
     float s, si;
     grid_dependency_wait();
