@@ -754,8 +754,8 @@ def run_ours(args, world, rank, local):
                                  "frac_of_tensor_pipe_rate": clock_normalised(a_sus, device_mhz_median),
                                  "probes": len(device_mhz), "sm_mhz_on_device_min_max": [round(device_mhz[0], 1), round(device_mhz[-1], 1)] if device_mhz else None,
                                  "sm_mhz_sampled_median": sus_clocks["sm_mhz"], "frac_with_sampled_clock": clock_normalised(a_sus, sus_clocks["sm_mhz"]),
-                                 "formula": "flop / (%d SMs x %d MAC x 2 x SM clock); the clock is read on the device by a one-warp probe kernel running "
-                                            "beside the step (200 us windows); the nvidia-smi samples of the same loop are given for comparison"
+                                 "formula": "flop / (%d SMs x %d MAC x 2 x SM clock); the clock is read on the device by a one-warp probe kernel on a second "
+                                            "stream during the loop (200 us windows, on whichever SM has registers free); the nvidia-smi samples of the same loop are given for comparison"
                                             % (sms, FP8_MACS_PER_SM_PER_CLOCK)},
             "burst": {"achieved": round(a_burst, 1), "peak": round(fp8_burst, 1), "frac": round(a_burst / fp8_burst, 4),
                       "regime": "the %d timed steps (%.3f s), divided by 2 x %s bf16 burst cuBLAS TFLOP/s" % (args.steps, total_ms / 1e3, pk["source"]),
