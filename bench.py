@@ -650,8 +650,9 @@ def run_ours(args, world, rank, local):
     if rank == 0:
         sampler2.start()
     sus_events = []
-    # the SM clock as the kernels see it: a one-warp probe kernel on a second stream, a 200 us window every few steps
-    n_probes = 32
+    # the SM clock as the kernels see it: a one-warp probe kernel on a second stream, a 100 us window every few steps
+    # (few and short: while a window is open on an SM, a CTA that needs the whole register file waits for it)
+    n_probes = 16
     probe_out = torch.zeros(n_probes, 2, dtype=torch.int64, device=device)
     s_probe = torch.cuda.Stream()
     probe_every = max(1, n_sus // n_probes)
@@ -660,7 +661,7 @@ def run_ours(args, world, rank, local):
         step.run_timed(sus_events)
         if i % probe_every == 0 and i // probe_every < n_probes and i >= n_sus // 4:
             with torch.cuda.stream(s_probe):
-                api.fp8_sm_clock_probe(probe_out[i // probe_every], 200)
+                api.fp8_sm_clock_probe(probe_out[i // probe_every], 100)
     barrier()
     probes = [(int(c), int(t)) for c, t in probe_out.cpu().tolist() if t > 0]
     device_mhz = sorted(c * 1000.0 / t for c, t in probes)
@@ -755,7 +756,7 @@ def run_ours(args, world, rank, local):
                                  "probes": len(device_mhz), "sm_mhz_on_device_min_max": [round(device_mhz[0], 1), round(device_mhz[-1], 1)] if device_mhz else None,
                                  "sm_mhz_sampled_median": sus_clocks["sm_mhz"], "frac_with_sampled_clock": clock_normalised(a_sus, sus_clocks["sm_mhz"]),
                                  "formula": "flop / (%d SMs x %d MAC x 2 x SM clock); the clock is read on the device by a one-warp probe kernel on a second "
-                                            "stream during the loop (200 us windows, on whichever SM has registers free); the nvidia-smi samples of the same loop are given for comparison"
+                                            "stream during the loop (100 us windows, on whichever SM has registers free); the nvidia-smi samples of the same loop are given for comparison"
                                             % (sms, FP8_MACS_PER_SM_PER_CLOCK)},
             "burst": {"achieved": round(a_burst, 1), "peak": round(fp8_burst, 1), "frac": round(a_burst / fp8_burst, 4),
                       "regime": "the %d timed steps (%.3f s), divided by 2 x %s bf16 burst cuBLAS TFLOP/s" % (args.steps, total_ms / 1e3, pk["source"]),
