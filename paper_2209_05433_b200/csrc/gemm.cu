@@ -23,7 +23,7 @@
 //                The epilogue of tile i overlaps the main loop of tile i+1.
 // Operands may be K-major or MN-major (forward / dgrad / wgrad layouts); the
 // two formats of a mixed E5M2 x E4M3 product are set in the instruction
-// descriptor.  No TMA load uses cluster multicast.
+// descriptor.  Every TMA load has one destination: the shared memory of the CTA that issues it.
 // Every mbarrier wait is bounded (about 2 s): on expiry the kernel latches an error code,
 // all roles drain, TMEM is freed and the kernel returns.
 #include <cuda.h>
