@@ -47,3 +47,21 @@ def sharded_amax_scale_quantize(x_local: torch.Tensor, fmt: int, out_local: torc
     api.fp8_scale_from_amax(a, fmt, s, si)
     api.fp8_quantize(x_local, fmt, s, out_local)
     return s, si
+
+
+def column_shard(n_cols: int, rank: int, world: int) -> tuple[int, int]:
+    """Columns [lo, hi) of a [rows, n_cols] weight or output owned by `rank`: boundaries are multiples of 16 columns,
+    so that a shard of FP8 codes (1 byte per element) and of the bf16 / fp32 output both start on 16 bytes."""
+    return shard_range(n_cols, rank, world, align=16)
+
+
+def column_parallel_gemm(A, fmt_a, major_a, B_local, fmt_b, major_b, D_local, sa_inv, sb_inv, amax_d, group=None, **kw):
+    """A product whose B operand (the weights of a forward layer) and output are split by output column across
+    ranks: D[:, lo:hi] = A . B[:, lo:hi].  Every rank holds all of A and its own columns of B and D (views with the
+    full row pitch are fine), so the contraction needs no exchange at all; the one per-tensor quantity of the whole
+    output, the epilogue amax the next scale factor is chosen from, is the MAX over the ranks' amax values: the same
+    4-byte all-reduce as for a sharded cast.  `amax_d` receives the amax of the WHOLE output on every rank."""
+    from . import api
+    api.fp8_gemm(A, fmt_a, major_a, B_local, fmt_b, major_b, D_local, sa_inv, sb_inv, amax_out=amax_d, **kw)
+    allreduce_amax_(amax_d, group)
+    return amax_d

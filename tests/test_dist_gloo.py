@@ -66,3 +66,12 @@ def test_shard_range_partitions_exactly():
             assert spans[0][0] == 0 and spans[-1][1] == n
             for (a, b), (c, d) in zip(spans[:-1], spans[1:]):
                 assert b == c and a <= b and (b % 16 == 0 or b == n)
+
+
+def test_column_shards_partition_the_output_columns_on_16_byte_boundaries():
+    for cols in (16, 1008, 4096, 49152, 12345):
+        for world in (1, 2, 3, 8):
+            spans = [fdist.column_shard(cols, r, world) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == cols
+            for (a, b), (c, d) in zip(spans[:-1], spans[1:]):
+                assert b == c and a <= b and (b % 16 == 0 or b == cols)

@@ -68,3 +68,59 @@ def test_two_ranks_quantize_one_tensor_with_one_scale(special, fmt):
         same_amax, same_scale, same_inv, same_codes, _ = ret[rank]
         assert same_amax and same_scale and same_inv and same_codes, (rank, ret[rank])
     assert ret[0][4][1] == ret[1][4][0] and ret[0][4][0] == 0 and ret[1][4][1] == n
+
+
+def _worker_columns(rank, world, port, ret):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        import oracle
+        from paper_2209_05433_b200 import api, synth
+        from paper_2209_05433_b200 import dist as fdist
+        from tests._util import THREADS, check_gemm_bf16, to_np_bits
+        torch.cuda.set_device(0)
+        T, I, O = 384, 2304, 1008                                        # K spans two 2048-chunks; O is not a multiple of the tile
+        X = synth.activations(T * I, 31, dtype=torch.bfloat16).view(T, I)
+        W = synth.weights(I * O, 32, 0.02, dtype=torch.bfloat16).view(I, O)
+        W[5, O - 3] = 40.0                                               # the largest output sits in the last rank's columns
+        xb, wb = to_np_bits(X).reshape(-1), to_np_bits(W).reshape(-1)
+        sx, six = oracle.scale_from_amax(oracle.amax(xb), oracle.E4M3)
+        sw, siw = oracle.scale_from_amax(oracle.amax(wb), oracle.E4M3)
+        Xq = oracle.quantize(xb, sx, oracle.E4M3).reshape(T, I)
+        Wq = oracle.quantize(wb, sw, oracle.E4M3).reshape(I, O)
+        lo, hi = fdist.column_shard(O, rank, world)
+        Xd, Wd = torch.from_numpy(Xq).cuda(), torch.from_numpy(Wq).cuda()          # every rank holds the whole tensors here; it
+        Y = torch.zeros(T, O, dtype=torch.bfloat16, device="cuda")                  # touches only its own columns of W and Y
+        sc = torch.tensor([six, siw, 0.0], dtype=torch.float32, device="cuda")
+        fdist.column_parallel_gemm(Xd, api.E4M3, api.MAJOR_K, Wd[:, lo:hi], api.E4M3, api.MAJOR_MN, Y[:, lo:hi], sc[0:1], sc[1:2], sc[2:3])
+        torch.cuda.synchronize()
+        assert api.fp8_async_status() == (0, 0)
+        ref, sab = oracle.gemm_rows(Xq, oracle.E4M3, (I, 1), Wq, oracle.E4M3, (O, 1), O, I, 0, T, six, siw, threads=THREADS)
+        got = to_np_bits(Y).reshape(T, O)
+        ok, _ = check_gemm_bf16(got[:, lo:hi], ref[:, lo:hi], sab[:, lo:hi], oracle.round_bf16_from_f64)
+        untouched = bool((np.delete(got, np.s_[lo:hi], axis=1) == 0).all())
+        # amax of the WHOLE output as stored: the other rank's columns are rounded from the oracle's reference (the two
+        # may differ by the accumulation tolerance, so compare with a tolerance of one bf16 step of the maximum)
+        whole = oracle.round_bf16_from_f64(ref).astype(np.uint16).reshape(T, O).copy()
+        whole[:, lo:hi] = got[:, lo:hi]
+        want = int(((whole & 0x7FFF).max()).astype(np.uint32)) << 16
+        got_amax = int(sc[2:3].cpu().numpy().view(np.uint32)[0])
+        ret[rank] = (bool(ok.all()), untouched, abs(got_amax - want) <= (1 << 16), got_amax, (lo, hi))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_split_the_output_columns_of_a_forward_product():
+    """column-parallel forward product: no exchange in the contraction, one 4-byte MAX all-reduce for the amax"""
+    world = 2
+    port = _free_port()
+    manager = mp.Manager()
+    ret = manager.dict()
+    mp.spawn(_worker_columns, args=(world, port, ret), nprocs=world, join=True)
+    assert len(ret) == world
+    for rank in range(world):
+        in_tolerance, untouched, amax_ok, _, _ = ret[rank]
+        assert in_tolerance and untouched and amax_ok, (rank, ret[rank])
+    assert ret[0][3] == ret[1][3]                                        # every rank ends with the same amax
+    assert ret[0][4][0] == 0 and ret[0][4][1] == ret[1][4][0] and ret[1][4][1] == 1008 and ret[0][4][1] % 16 == 0
