@@ -108,3 +108,32 @@ def test_gemm_with_per_channel_weight_scales(out_dtype, shape):
     a2 = _scalar(-1.0)
     api.fp8_amax(D.contiguous(), a2)
     assert amax_d.cpu().numpy().view(np.uint32)[0] == a2.cpu().numpy().view(np.uint32)[0]
+
+
+def test_quantize_per_column_at_the_size_where_the_slabs_become_short():
+    """From 256 MB on the per-column conversion runs 64-row slabs: a tensor just above that size, with a row count that
+    is no multiple of the slab, a row pitch wider than the row, and special values, against the oracle bit for bit;
+    the bytes around the output stay untouched."""
+    rows, cols, pitch = 16400 + 37, 8192, 8208                      # 269 MB of bf16
+    base = synth.weights(rows * pitch, 17, 0.02, dtype=torch.bfloat16, device=DEV)
+    x = base.view(rows, pitch)[:, :cols]
+    x[rows - 1, cols - 1] = float("nan")
+    x[rows - 2, 3] = float("inf")
+    x[77, 4100] = 11.0
+    x_np = to_np_bits(x)
+    amax = torch.empty(cols, dtype=torch.float32, device=DEV)
+    api.fp8_amax_channels(x, 0, amax)
+    want_amax = oracle.amax_channels(x_np, 0)
+    assert np.array_equal(amax.cpu().numpy().view(np.uint32), want_amax.view(np.uint32))
+    s, si = torch.empty(cols, dtype=torch.float32, device=DEV), torch.empty(cols, dtype=torch.float32, device=DEV)
+    api.fp8_scales_from_amax(amax, E4, s, si)
+    ws, _ = oracle.scales_from_amax(want_amax, E4)
+    out_full = torch.full((rows + 1, cols + 16), 0xA5, dtype=torch.uint8, device=DEV)
+    out = out_full[:rows, :cols]
+    api.fp8_quantize_channels(x, 0, E4, s, out)
+    torch.cuda.synchronize()
+    want = oracle.quantize_channels(x_np, ws, 0, E4, api.SATURATE)
+    got = out.cpu().numpy()
+    bad = np.argwhere(got != want)
+    assert bad.size == 0, bad[:5].tolist()
+    assert bool((out_full[rows:, :] == 0xA5).all()) and bool((out_full[:rows, cols:] == 0xA5).all())
