@@ -1363,6 +1363,15 @@ static int grid_for(int64_t work_items) {
     return (int)g;
 }
 
+// One warp per unit of work, every unit its own short-lived warp: the hardware scheduler hands the blocks out in index order
+// and evens out what an equal static share per resident block cannot (see the flat kernels).
+static int grid_one_warp_per_unit(int64_t units) {
+    int64_t g = (units * 32 + kThreads - 1) / kThreads;
+    if (g > 0x7FFFFFFF) g = 0x7FFFFFFF;                  // the kernels stride over what is left
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
 // segments per row of the row kernels: 32 lanes x kRowsUnroll items each, at least one
 static int64_t row_segments(int64_t n_items) {
     const int64_t per = 32 * kRowsUnroll;
@@ -1403,7 +1412,7 @@ static fp8_status launch_amax_channels(const void* x, int64_t rows, int64_t cols
             if (cudaMemsetAsync(bits, 0, (size_t)channels * 4, st) != cudaSuccess) return FP8_ERR_CUDA;
             count_launches(1);
         }
-        k_amax_rows<WIDE><<<grid_for(rows * segs * 32), kThreads, 0, st>>>(x, rows, cols, ld, segs, span, bits);
+        k_amax_rows<WIDE><<<grid_one_warp_per_unit(rows * segs), kThreads, 0, st>>>(x, rows, cols, ld, segs, span, bits);
         count_launches(1);
         return launch_status();
     }
@@ -1431,7 +1440,7 @@ static fp8_status launch_quantize_channels(const void* x, int64_t rows, int64_t 
     const bool vec = aligned16(x) && ((ld * ESZ) & 15) == 0 && (reinterpret_cast<uintptr_t>(out) & (EPI - 1)) == 0 && (ld_out % EPI) == 0;
     if (vec && axis == 1) {
         const int64_t segs = row_segments(cols / EPI);
-        k_quantize_rows<WIDE, FMT, NOSAT><<<grid_for(rows * segs * 32), kThreads, 0, st>>>(x, rows, cols, ld, segs, scale, out, ld_out);
+        k_quantize_rows<WIDE, FMT, NOSAT><<<grid_one_warp_per_unit(rows * segs), kThreads, 0, st>>>(x, rows, cols, ld, segs, scale, out, ld_out);
         count_launches(1);
         return launch_status();
     }
