@@ -1151,9 +1151,12 @@ constexpr int kFakeUnroll = 2;
 template <int WIDE>
 static fp8_status launch_amax(const void* x, size_t n, uint32_t* bits, cudaStream_t st) {
     if (aligned16(x)) {
-        auto k = k_amax<WIDE, kAmaxUnroll>;
-        const int grid = stream_grid(chunks_of(n, WIDE == kWideBF16 ? 8 : 4, kAmaxUnroll), kAmaxChunksPerBlock);
-        if (launch_programmatic(k, dim3(grid), dim3(kThreads), st, x, n, bits) != cudaSuccess) return FP8_ERR_CUDA;
+        constexpr int EPI = WIDE == kWideBF16 ? 8 : 4;
+        const bool small = n * (WIDE == kWideBF16 ? 2 : 4) <= ((size_t)64 << 20);     // half-size chunks, as in launch_quantize
+        const cudaError_t e = small
+            ? launch_programmatic(k_amax<WIDE, kAmaxUnroll / 2>, dim3(stream_grid(chunks_of(n, EPI, kAmaxUnroll / 2), kAmaxChunksPerBlock)), dim3(kThreads), st, x, n, bits)
+            : launch_programmatic(k_amax<WIDE, kAmaxUnroll>, dim3(stream_grid(chunks_of(n, EPI, kAmaxUnroll), kAmaxChunksPerBlock)), dim3(kThreads), st, x, n, bits);
+        if (e != cudaSuccess) return FP8_ERR_CUDA;
     } else {
         auto k = k_amax_elementwise<WIDE>;
         const int grid = stream_grid((n + kThreads - 1) / kThreads, 16);
